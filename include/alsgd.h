@@ -1,0 +1,242 @@
+/*
+ * alsgd.h — C ABI of the asynchronous Local-SGD server step and the workers' inner AdamW step,
+ * on one NVIDIA B200 (sm_100a).
+ *
+ * The library keeps, in one caller-owned device arena, the server state of the paper's Algorithm 3
+ * ("Delayed Nesterov": global parameters theta, momentum m, buffer Delta, update counter t) and W
+ * simulated workers (fp32 parameters, the fp32 snapshot they were dispatched with, AdamW moments,
+ * a bf16 replica), all as flat vectors of P elements laid out from a tensor table.
+ *
+ * Conventions
+ *   - Every function returns ALSGD_OK (0) or a negative alsgd_status.  Nothing throws, aborts,
+ *     traps or prints.  On an error the context is left as it was before the call.
+ *   - "host" / "device" is stated for every pointer.  The arena and the stream belong to the
+ *     caller; the context owns only host bookkeeping.  No entry point allocates device memory
+ *     (alsgd_init and alsgd_destroy allocate and free host memory only).
+ *   - Calls enqueue work on the context's stream and return without waiting, except where a
+ *     host output needs the result (stated per call).  A context is not thread-safe.
+ *   - All element counts and indices are 64-bit.
+ */
+#ifndef ALSGD_H
+#define ALSGD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum alsgd_status {
+    ALSGD_OK = 0,
+    ALSGD_E_ARG = -1,    /* invalid argument (null pointer, zero size, value outside its domain) */
+    ALSGD_E_RANGE = -2,  /* worker id or index out of range */
+    ALSGD_E_STATE = -3,  /* call not allowed in the current state (e.g. arrival of a worker never dispatched) */
+    ALSGD_E_CUDA = -4,   /* a CUDA runtime call failed; see alsgd_last_cuda_error */
+    ALSGD_E_NOMEM = -5,  /* arena too small, or host allocation failed */
+    ALSGD_E_UNSUPPORTED = -6
+} alsgd_status;
+
+/* Text for a status code (static storage, host). */
+const char* alsgd_strerror(int status);
+
+/* ------------------------------------------------------------------------------------------------
+ * Flat-buffer layout.  The paper treats the model as one parameter vector theta (Algorithm 3 acts
+ * on it elementwise); the tensor table only says where each tensor lives in that vector and whether
+ * the inner optimizer applies weight decay to it (Table 5: weight decay 0.1).
+ * ---------------------------------------------------------------------------------------------- */
+#define ALSGD_TENSOR_DECAY 1u
+
+typedef struct alsgd_tensor_desc {
+    uint64_t numel;   /* > 0 */
+    uint32_t flags;   /* ALSGD_TENSOR_DECAY or 0 */
+    uint32_t reserved;
+} alsgd_tensor_desc;
+
+/* Offsets of n tensors in the flat vector: tensor i starts at the next multiple of align_elems
+ * (>= 1) after tensor i-1; *P_out is the padded total (a multiple of align_elems).  Padding
+ * elements are zero, are never weight-decayed and take part in nothing observable.
+ * tensors: host, n entries.  offsets_out: host, n entries, may be NULL.  ALSGD_E_ARG on n = 0,
+ * numel = 0, align_elems = 0 or 64-bit overflow. */
+int alsgd_layout_size(const alsgd_tensor_desc* tensors, uint32_t n, uint32_t align_elems,
+                      uint64_t* P_out, uint64_t* offsets_out);
+
+/* ------------------------------------------------------------------------------------------------
+ * Context
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct alsgd_ctx alsgd_ctx;
+
+/* Which model the pseudo-gradient of an arriving worker is taken against. */
+#define ALSGD_PG_DISPATCH 0u  /* the model the worker was seeded with: delta = theta^(t-1) - theta_i (Algorithm 1) */
+#define ALSGD_PG_CURRENT 1u   /* the running global model at the moment of that arrival */
+
+#define ALSGD_CFG_REPLICA_BF16 1u  /* keep a bf16 copy of every worker's parameters */
+#define ALSGD_CFG_GRAD_STAGING 2u  /* reserve a P-element fp32 staging buffer so that alsgd_inner_adamw accepts host gradients */
+
+typedef struct alsgd_config {
+    uint32_t n_workers;  /* W >= 1 replicas resident in the arena */
+    uint32_t N;          /* Algorithm 3 buffer size (the "delay period" of Table 5), >= 1 */
+    uint32_t pg_base;    /* ALSGD_PG_DISPATCH or ALSGD_PG_CURRENT */
+    uint32_t flags;      /* ALSGD_CFG_* */
+    float beta;          /* momentum decay, [0, 1) */
+    float outer_lr;      /* epsilon of Algorithm 3 */
+    float c;             /* momentum activation, [0, 1/N] (Algorithm 3; default 0) */
+    float adam_b1, adam_b2, adam_eps, adam_wd; /* inner AdamW: betas in [0,1), eps >= 0, wd >= 0 */
+    int32_t device;      /* CUDA device ordinal that owns arena and stream */
+    void* stream;        /* cudaStream_t (0 = legacy default stream); caller-owned */
+    void* arena;         /* device, 256-byte aligned, caller-owned for the context's lifetime */
+    uint64_t arena_bytes;
+} alsgd_config;
+
+/* Bytes of arena needed for a layout and configuration (pure host arithmetic). */
+int alsgd_arena_bytes(const alsgd_tensor_desc* tensors, uint32_t n, uint32_t align_elems,
+                      const alsgd_config* cfg, uint64_t* bytes_out);
+
+/* Create a context in the state Algorithm 3 starts from: t = 0, m = 0, Delta = 0; theta = 0 until
+ * alsgd_set_global; every worker is "never dispatched" with zero AdamW moments.  Enqueues the zero
+ * fills on cfg->stream.  ALSGD_E_ARG for values outside the domains above or a misaligned arena,
+ * ALSGD_E_NOMEM if arena_bytes is too small. */
+int alsgd_init(alsgd_ctx** out, const alsgd_tensor_desc* tensors, uint32_t n, uint32_t align_elems,
+               const alsgd_config* cfg);
+
+/* Free the host bookkeeping.  Never touches the arena.  Does not wait for the stream. */
+int alsgd_destroy(alsgd_ctx* ctx);
+
+/* Load theta^(0) (Algorithm 2: theta <- theta^(0)) / read theta.  P floats; is_device says where the
+ * caller's buffer lives.  Host buffers: the copy is enqueued and the call waits for it. */
+int alsgd_set_global(alsgd_ctx* ctx, const float* src, int src_is_device);
+int alsgd_get_global(alsgd_ctx* ctx, float* dst, int dst_is_device);
+
+/* Overwrite / read one worker's fp32 parameters (a test and simulation hook: it stands in for the
+ * forward/backward passes this library does not run).  Same pointer rules as alsgd_set_global. */
+int alsgd_set_worker_params(alsgd_ctx* ctx, uint32_t worker, const float* src, int src_is_device);
+int alsgd_get_worker_params(alsgd_ctx* ctx, uint32_t worker, float* dst, int dst_is_device);
+
+/* Dispatch one worker with the current server model (Algorithm 2, train(W, theta); Algorithm 1,
+ * theta_i <- theta): its parameters, its dispatch snapshot and its bf16 replica become theta; its
+ * pull tick becomes t.  AdamW moments and step count are untouched (the paper keeps the inner
+ * optimizer state on the worker across rounds and never resets it).  ALSGD_E_RANGE for a bad id. */
+int alsgd_pull(alsgd_ctx* ctx, uint32_t worker);
+
+/* One inner AdamW step of one worker (InnerOpt of Algorithm 1; decoupled weight decay on tensors
+ * flagged ALSGD_TENSOR_DECAY, bias correction from `step`, epsilon outside the root), followed by
+ * the bf16 cast of the new parameters into the replica.
+ *   grads            P fp32 values, 16-byte aligned, device or host (host needs
+ *                    ALSGD_CFG_GRAD_STAGING; the copy is enqueued on the stream and the buffer is
+ *                    borrowed until the stream reaches it)
+ *   step             the worker's lifetime step count, >= 1
+ *   lr               learning rate of this step
+ * ALSGD_E_STATE if the worker was never dispatched, ALSGD_E_ARG if step = 0. */
+int alsgd_inner_adamw(alsgd_ctx* ctx, uint32_t worker, const float* grads, int grads_is_device,
+                      uint64_t step, float lr);
+
+#define ALSGD_ARRIVE_RESEED 1u    /* re-dispatch all k workers with the final theta (Algorithm 2, the branch taken when get_worker() finds nobody) */
+#define ALSGD_ARRIVE_NORM 2u      /* report the squared norm of each pseudo-gradient */
+#define ALSGD_ARRIVE_NANCHECK 4u  /* report whether each pseudo-gradient has a non-finite entry */
+
+typedef struct alsgd_arrival_info {
+    uint64_t tick;       /* Algorithm 3's t at which this arrival was applied */
+    uint64_t staleness;  /* tick minus the worker's pull tick */
+    double gnorm2;       /* sum of squared pseudo-gradient entries (0 unless NORM) */
+    uint32_t worker;
+    uint32_t boundary;   /* 1 if (t+1) % N == 0: momentum updated, buffer reset */
+    uint32_t nonfinite;  /* 1 if any entry was NaN or Inf (0 unless NANCHECK) */
+    uint32_t reserved;
+} alsgd_arrival_info;
+
+/* The sync() of Algorithm 2 for the k workers of one grace window, in the given order: for each,
+ * pseudo-gradient -> Delta += g -> on every N-th server update m <- beta m + Delta/N,
+ * theta <- theta - eps((1-cN+c) beta m + g/N), Delta <- 0; otherwise theta <- theta - eps(c beta m + g/N)
+ * (Algorithm 3); t advances by k.  The k arrivals are applied in one pass over memory and give
+ * exactly the result of k single calls.  With RESEED all k workers are then dispatched again with
+ * the final theta.
+ *   worker_ids   host, k entries, copied at call time
+ *   info         host, k entries or NULL.  With NORM or NANCHECK and info != NULL the call waits for
+ *                the stream; otherwise it only enqueues.
+ * k = 0 is a no-op.  ALSGD_E_ARG: k > W, a duplicate id.  ALSGD_E_RANGE: id >= W.  ALSGD_E_STATE: a
+ * worker that is not currently dispatched (never pulled, or already arrived and not re-dispatched). */
+int alsgd_arrive(alsgd_ctx* ctx, const uint32_t* worker_ids, uint32_t k, uint32_t flags,
+                 alsgd_arrival_info* info);
+
+/* Server update counter t of Algorithm 3 and its phase t % N.  Either pointer may be NULL. */
+int alsgd_counters(alsgd_ctx* ctx, uint64_t* t_out, uint32_t* phase_out);
+
+typedef struct alsgd_ptrs {
+    float* theta;  /* device, P */
+    float* m;      /* device, P */
+    float* delta;  /* device, P */
+    uint64_t P;
+    uint32_t n_workers;
+    uint32_t reserved;
+} alsgd_ptrs;
+
+typedef struct alsgd_worker_ptrs {
+    float* p;          /* device, P: the worker's parameters */
+    float* base;       /* device, P: dispatch snapshot (NULL in ALSGD_PG_CURRENT mode) */
+    float* adam_m;     /* device, P */
+    float* adam_v;     /* device, P */
+    uint16_t* replica; /* device, P bf16 bit patterns (NULL without ALSGD_CFG_REPLICA_BF16) */
+} alsgd_worker_ptrs;
+
+/* Borrowed device pointers into the arena, valid until alsgd_destroy, for a harness that perturbs
+ * workers and reads results.  Right after a momentum boundary Delta is zero by definition and the
+ * library may not have written those zeros yet; this call enqueues that fill first, so every read
+ * ordered after it on the context's stream sees Algorithm 3's Delta. */
+int alsgd_state_ptrs(alsgd_ctx* ctx, alsgd_ptrs* out);
+int alsgd_worker_state_ptrs(alsgd_ctx* ctx, uint32_t worker, alsgd_worker_ptrs* out);
+
+/* Wait for the context's stream. */
+int alsgd_sync(alsgd_ctx* ctx);
+
+/* cudaError_t of the most recent failed CUDA call of this context (0 if none). */
+int alsgd_last_cuda_error(alsgd_ctx* ctx);
+
+/* ------------------------------------------------------------------------------------------------
+ * Host-side helpers of the method (no device work)
+ * ---------------------------------------------------------------------------------------------- */
+
+/* Dynamic Local Updates, Eq. 6: steps_w = floor(v_w / max v * H), at least 1.
+ * speeds: host, n positive values (steps per second).  steps_out: host, n entries. */
+int alsgd_dylu_steps(const double* speeds, uint32_t n, uint32_t H, uint32_t* steps_out);
+
+typedef struct alsgd_lr_sched {
+    double eta_max, eta_min;
+    uint64_t t_warmup, T;
+} alsgd_lr_sched;
+
+/* Learning rate of Eq. 3 at shard-local step t: linear warm-up, then cosine decay to eta_min with
+ * the ratio (t - t_warmup)/(T - t_warmup) kept inside [0, 1] and T - t_warmup >= 0. */
+int alsgd_lr_at(const alsgd_lr_sched* sched, uint64_t t, double* lr_out);
+
+/* Asynchronous task scheduling (Algorithm 2 with get_worker() of Algorithm 5) on faked time.
+ * The caller plays train(): it dispatches a job for a worker with the time that job will take;
+ * alsgd_sched_next_batch returns the workers the server synchronises in one grace window, in order. */
+typedef struct alsgd_sched alsgd_sched;
+
+/* tau_grace >= 0.  t_max: total local updates after which no further arrival is produced (0 = no limit). */
+int alsgd_sched_create(alsgd_sched** out, uint32_t n_workers, double tau_grace, uint64_t t_max);
+int alsgd_sched_destroy(alsgd_sched* s);
+
+/* Start a job on an idle worker.  It starts at time 0 if the worker has never run, else at the moment
+ * the grace window that synchronised it closed (tau_sync + tau_grace), and completes `duration`
+ * (> 0) later; `local_updates` is added to t_local when it is synchronised.
+ * ALSGD_E_STATE if the worker already has a job in flight. */
+int alsgd_sched_dispatch(alsgd_sched* s, uint32_t worker, double duration, uint32_t local_updates);
+
+/* Run Algorithm 2's loop until get_worker() returns null: collect the earliest completed worker (ties:
+ * lower id) while its completion time is within tau_grace of the window's first, then close the window.
+ *   ids_out, times_out   host, cap entries (times_out may be NULL)
+ *   k_out                number of workers in the window (0 once t_local >= t_max)
+ *   restart_out          time at which the returned workers start their next job (may be NULL)
+ * The returned workers are idle until dispatched again.  ALSGD_E_STATE if no job is in flight,
+ * ALSGD_E_NOMEM if cap is smaller than the window (nothing is consumed). */
+int alsgd_sched_next_batch(alsgd_sched* s, uint32_t* ids_out, double* times_out, uint32_t cap,
+                           uint32_t* k_out, double* restart_out);
+
+/* Total local updates synchronised so far (Algorithm 2's t_local). */
+int alsgd_sched_local_updates(alsgd_sched* s, uint64_t* t_local_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ALSGD_H */

@@ -1,0 +1,59 @@
+// Internal launch interface between the host-side context and the sm_100a kernels.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace alsgd {
+
+constexpr int kMaxArrivals = 8;  // arrivals folded into one pass over theta / Delta / m
+constexpr int kMaxSeeds = 8;     // replicas re-seeded by one launch
+
+enum : uint32_t {
+    kDeltaZeroIn = 1u,     // Delta is zero by definition on entry: do not read it
+    kDeltaSkipStore = 2u,  // Delta is zero by definition on exit: do not write it
+    kReadM = 4u,           // momentum is needed (a boundary in the batch, or c != 0)
+    kWriteM = 8u,          // momentum changes (a boundary in the batch)
+    kCNonZero = 16u        // momentum activation c != 0
+};
+
+// One batch of arrivals of Algorithm 3 plus the re-seed of the workers that are dispatched again.
+struct ArriveArgs {
+    float* theta;
+    float* delta;
+    float* mom;
+    const float* base[kMaxArrivals];  // dispatch snapshots (unused when the pseudo-gradient is against running theta)
+    const float* p[kMaxArrivals];     // arriving workers' parameters
+    float* seed_p[kMaxSeeds];
+    float* seed_base[kMaxSeeds];      // may be null
+    uint16_t* seed_rep[kMaxSeeds];    // may be null
+    double* gnorm2;                   // scratch: kMaxArrivals accumulators, zeroed by the caller
+    unsigned int* nonfinite;          // scratch: kMaxArrivals flags, zeroed by the caller
+    uint64_t n;                       // elements
+    uint32_t n_arr;
+    uint32_t n_seed;
+    uint32_t boundary_mask;           // bit j: arrival j is a momentum boundary
+    uint32_t flags;
+    float beta, eps, inv_n, cb, cn;
+};
+
+struct AdamArgs {
+    float* p;
+    float* m;
+    float* v;
+    const float* g;
+    uint16_t* rep;             // may be null
+    const uint64_t* seg_end;   // device: ascending exclusive end of each weight-decay segment; last == n
+    const uint32_t* seg_decay; // device: 1 if the segment is weight-decayed
+    uint32_t n_seg;
+    uint64_t n;
+    float b1, b2, omb1, omb2, bc1, bc2, eps, lr, wd;
+};
+
+struct LaunchCfg {
+    int sm_count;
+};
+
+cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, const LaunchCfg& lc, cudaStream_t s);
+cudaError_t launch_adamw(const AdamArgs& a, const LaunchCfg& lc, cudaStream_t s);
+
+}  // namespace alsgd
