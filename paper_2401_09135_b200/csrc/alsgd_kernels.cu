@@ -1,0 +1,368 @@
+// sm_100a kernels of the asynchronous Local-SGD server step and the inner AdamW step.
+//
+// Every kernel here is a pure stream over flat fp32 vectors (0.3-0.6 flop per byte), so the design
+// goal is HBM bandwidth: 128-bit coalesced accesses, several independent vectors in flight per
+// thread, touch-once cache hints, one pass over theta / Delta / m no matter how many workers
+// arrive, and the re-seed of the dispatched workers written from registers in the same pass.
+//
+// Arithmetic contract: every fp32 operation is a separate IEEE-754 round-to-nearest operation in
+// the order Algorithm 3 states it (this file is compiled with -fmad=false, IEEE division and
+// square root, no flush-to-zero), so results do not depend on the launch shape.
+#include "alsgd_kernels.cuh"
+
+#include <cuda_runtime.h>
+
+namespace alsgd {
+
+namespace {
+
+constexpr int kBlock = 256;
+
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
+__device__ __forceinline__ void st_stream(uint2* p, uint2 v) { __stcs(p, v); }
+
+// bf16 round-to-nearest-even on the raw bits; NaN becomes a quiet NaN with the sign kept.
+__device__ __forceinline__ uint32_t bf16_bits(float x) {
+    const uint32_t u = __float_as_uint(x);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return ((u >> 16) & 0x8000u) | 0x7FC0u;
+    return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+}
+
+__device__ __forceinline__ uint2 bf16_pack4(const float4& x) {
+    uint2 r;
+    r.x = bf16_bits(x.x) | (bf16_bits(x.y) << 16);
+    r.y = bf16_bits(x.z) | (bf16_bits(x.w) << 16);
+    return r;
+}
+
+// K sequential arrivals of Algorithm 3 on one element.  th, d, mm carry theta, Delta, momentum.
+template <int K, bool DIAG, bool CUR>
+__device__ __forceinline__ void dn_element(float& th, float& d, float& mm, const float* b, const float* p,
+                                           const ArriveArgs& a, double* acc, uint32_t& bad) {
+#pragma unroll
+    for (int j = 0; j < K; ++j) {
+        const float start = CUR ? th : b[j];
+        const float g = start - p[j];                 // pseudo-gradient
+        if (DIAG) {
+            acc[j] += (double)g * (double)g;
+            if (!isfinite(g)) bad |= 1u << j;
+        }
+        d = d + g;                                    // Delta <- Delta + g
+        const float gn = g * a.inv_n;                 // g / N
+        if ((a.boundary_mask >> j) & 1u) {
+            const float mn = (a.beta * mm) + (d * a.inv_n);   // m <- beta m + Delta/N
+            const float u = (a.cb * mn) + gn;                 // (1-cN+c) beta m + g/N
+            th = th - (a.eps * u);
+            mm = mn;
+            d = 0.0f;
+        } else {
+            const float u = (a.flags & kCNonZero) ? ((a.cn * mm) + gn) : gn;   // c beta m + g/N
+            th = th - (a.eps * u);
+        }
+    }
+}
+
+template <int K, int V, bool DIAG, bool CUR>
+__global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ ArriveArgs a) {
+    constexpr int KK = K > 0 ? K : 1;
+    const uint64_t nvec = a.n >> 2;
+    const uint64_t tile = (uint64_t)kBlock * V;
+    const uint32_t flags = a.flags;
+    const bool read_delta = K > 0 && !(flags & kDeltaZeroIn);
+    const bool write_delta = K > 0 && !(flags & kDeltaSkipStore);
+    const bool read_m = K > 0 && (flags & kReadM);
+    const bool write_m = K > 0 && (flags & kWriteM);
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    double acc[KK];
+    uint32_t bad = 0;
+#pragma unroll
+    for (int j = 0; j < KK; ++j) acc[j] = 0.0;
+
+    float4* __restrict__ theta4 = reinterpret_cast<float4*>(a.theta);
+    float4* __restrict__ delta4 = reinterpret_cast<float4*>(a.delta);
+    float4* __restrict__ mom4 = reinterpret_cast<float4*>(a.mom);
+
+    for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < nvec; t0 += (uint64_t)gridDim.x * tile) {
+        float4 th[V], d[V], mm[V];
+        float4 b[KK][V], p[KK][V];
+        // ---- issue every load of the tile before the first use
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const uint64_t i = t0 + (uint64_t)v * kBlock + threadIdx.x;
+            const bool ok = i < nvec;
+            th[v] = ok ? ld_stream(theta4 + i) : zero4;
+            d[v] = (ok && read_delta) ? ld_stream(delta4 + i) : zero4;
+            mm[v] = (ok && read_m) ? ld_stream(mom4 + i) : zero4;
+#pragma unroll
+            for (int j = 0; j < K; ++j) {
+                p[j][v] = ok ? ld_stream(reinterpret_cast<const float4*>(a.p[j]) + i) : zero4;
+                if (!CUR) b[j][v] = ok ? ld_stream(reinterpret_cast<const float4*>(a.base[j]) + i) : zero4;
+            }
+        }
+        // ---- arithmetic and stores
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const uint64_t i = t0 + (uint64_t)v * kBlock + threadIdx.x;
+            if (i >= nvec) continue;
+            if (K > 0) {
+                float* thf = reinterpret_cast<float*>(&th[v]);
+                float* df = reinterpret_cast<float*>(&d[v]);
+                float* mf = reinterpret_cast<float*>(&mm[v]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float be[KK], pe[KK];
+#pragma unroll
+                    for (int j = 0; j < K; ++j) {
+                        pe[j] = reinterpret_cast<const float*>(&p[j][v])[e];
+                        be[j] = CUR ? 0.f : reinterpret_cast<const float*>(&b[j][v])[e];
+                    }
+                    dn_element<K, DIAG, CUR>(thf[e], df[e], mf[e], be, pe, a, acc, bad);
+                }
+                st_stream(theta4 + i, th[v]);
+                if (write_delta) st_stream(delta4 + i, d[v]);
+                if (write_m) st_stream(mom4 + i, mm[v]);
+            }
+            if (a.n_seed) {
+                const uint2 packed = bf16_pack4(th[v]);
+#pragma unroll
+                for (int s = 0; s < kMaxSeeds; ++s) {
+                    if (s < (int)a.n_seed) {
+                        st_stream(reinterpret_cast<float4*>(a.seed_p[s]) + i, th[v]);
+                        if (a.seed_base[s]) st_stream(reinterpret_cast<float4*>(a.seed_base[s]) + i, th[v]);
+                        if (a.seed_rep[s]) st_stream(reinterpret_cast<uint2*>(a.seed_rep[s]) + i, packed);
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- up to three trailing elements when n is not a multiple of four
+    const uint64_t rem0 = nvec << 2;
+    if (blockIdx.x == 0 && rem0 + threadIdx.x < a.n) {
+        const uint64_t i = rem0 + threadIdx.x;
+        float th = a.theta[i];
+        if (K > 0) {
+            float d = read_delta ? a.delta[i] : 0.f;
+            float mm = read_m ? a.mom[i] : 0.f;
+            float be[KK], pe[KK];
+#pragma unroll
+            for (int j = 0; j < K; ++j) {
+                pe[j] = a.p[j][i];
+                be[j] = CUR ? 0.f : a.base[j][i];
+            }
+            dn_element<K, DIAG, CUR>(th, d, mm, be, pe, a, acc, bad);
+            a.theta[i] = th;
+            if (write_delta) a.delta[i] = d;
+            if (write_m) a.mom[i] = mm;
+        }
+        for (uint32_t s = 0; s < a.n_seed; ++s) {
+            a.seed_p[s][i] = th;
+            if (a.seed_base[s]) a.seed_base[s][i] = th;
+            if (a.seed_rep[s]) a.seed_rep[s][i] = (uint16_t)bf16_bits(th);
+        }
+    }
+
+    // ---- optional diagnostics: one double atomic per block per arrival, one flag per arrival
+    if (DIAG && K > 0) {
+        __shared__ double warp_sum[kBlock / 32][KK];
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+        for (int j = 0; j < K; ++j) {
+            double s = acc[j];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xFFFFFFFFu, s, o);
+            if (lane == 0) warp_sum[warp][j] = s;
+        }
+        bad = __reduce_or_sync(0xFFFFFFFFu, bad);
+        if (lane == 0 && bad) {
+            for (int j = 0; j < K; ++j)
+                if ((bad >> j) & 1u) atomicOr(a.nonfinite + j, 1u);
+        }
+        __syncthreads();
+        if ((int)threadIdx.x < K) {
+            double s = 0.0;
+            for (int w = 0; w < kBlock / 32; ++w) s += warp_sum[w][threadIdx.x];
+            atomicAdd(a.gnorm2 + threadIdx.x, s);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Inner AdamW step with decoupled weight decay, fused with the bf16 cast of the new parameters.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void adam_element(float& p, float& m, float& v, float g, bool decay, const AdamArgs& a) {
+    const float mi = (a.b1 * m) + (a.omb1 * g);
+    const float vi = (a.b2 * v) + (a.omb2 * (g * g));
+    m = mi;
+    v = vi;
+    const float mh = mi / a.bc1;
+    const float vh = vi / a.bc2;
+    const float r = mh / (sqrtf(vh) + a.eps);
+    p = decay ? (p - (a.lr * (r + (a.wd * p)))) : (p - (a.lr * r));
+}
+
+struct SegCursor {
+    uint32_t idx;
+    uint64_t end;
+    uint32_t decay;
+};
+
+__device__ __forceinline__ void seg_seek(SegCursor& c, uint64_t e, const AdamArgs& a) {
+    while (e >= c.end && c.idx + 1 < a.n_seg) {
+        ++c.idx;
+        c.end = __ldg(a.seg_end + c.idx);
+        c.decay = __ldg(a.seg_decay + c.idx);
+    }
+}
+
+__device__ __forceinline__ SegCursor seg_find(uint64_t e, const AdamArgs& a) {
+    uint32_t lo = 0, hi = a.n_seg - 1;            // first segment whose end is > e
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (__ldg(a.seg_end + mid) > e) hi = mid; else lo = mid + 1;
+    }
+    SegCursor c;
+    c.idx = lo;
+    c.end = __ldg(a.seg_end + lo);
+    c.decay = __ldg(a.seg_decay + lo);
+    return c;
+}
+
+template <int V>
+__global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ AdamArgs a) {
+    const uint64_t nvec = a.n >> 2;
+    const uint64_t tile = (uint64_t)kBlock * V;
+    float4* __restrict__ p4 = reinterpret_cast<float4*>(a.p);
+    float4* __restrict__ m4 = reinterpret_cast<float4*>(a.m);
+    float4* __restrict__ v4 = reinterpret_cast<float4*>(a.v);
+    const float4* __restrict__ g4 = reinterpret_cast<const float4*>(a.g);
+    uint2* __restrict__ rep2 = reinterpret_cast<uint2*>(a.rep);
+
+    SegCursor cur;
+    bool have_cur = false;
+
+    for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < nvec; t0 += (uint64_t)gridDim.x * tile) {
+        float4 p[V], m[V], v[V], g[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            const uint64_t i = t0 + (uint64_t)k * kBlock + threadIdx.x;
+            if (i < nvec) {
+                g[k] = ld_stream(g4 + i);
+                p[k] = ld_stream(p4 + i);
+                m[k] = ld_stream(m4 + i);
+                v[k] = ld_stream(v4 + i);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            const uint64_t i = t0 + (uint64_t)k * kBlock + threadIdx.x;
+            if (i >= nvec) continue;
+            const uint64_t e0 = i << 2;
+            if (!have_cur) { cur = seg_find(e0, a); have_cur = true; }
+            seg_seek(cur, e0, a);
+            float* pf = reinterpret_cast<float*>(&p[k]);
+            float* mf = reinterpret_cast<float*>(&m[k]);
+            float* vf = reinterpret_cast<float*>(&v[k]);
+            const float* gf = reinterpret_cast<const float*>(&g[k]);
+            if (e0 + 4 <= cur.end) {
+                const bool dec = cur.decay != 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) adam_element(pf[e], mf[e], vf[e], gf[e], dec, a);
+            } else {                                   // the vector straddles a segment edge
+                SegCursor c = cur;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    seg_seek(c, e0 + e, a);
+                    adam_element(pf[e], mf[e], vf[e], gf[e], c.decay != 0, a);
+                }
+            }
+            st_stream(p4 + i, p[k]);
+            st_stream(m4 + i, m[k]);
+            st_stream(v4 + i, v[k]);
+            if (a.rep) st_stream(rep2 + i, bf16_pack4(p[k]));
+        }
+    }
+
+    const uint64_t rem0 = nvec << 2;
+    if (blockIdx.x == 0 && rem0 + threadIdx.x < a.n) {
+        const uint64_t i = rem0 + threadIdx.x;
+        SegCursor c = seg_find(i, a);
+        float p = a.p[i], m = a.m[i], v = a.v[i];
+        adam_element(p, m, v, a.g[i], c.decay != 0, a);
+        a.p[i] = p;
+        a.m[i] = m;
+        a.v[i] = v;
+        if (a.rep) a.rep[i] = (uint16_t)bf16_bits(p);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Launch shapes: persistent grids, a whole number of resident blocks per SM.
+// ---------------------------------------------------------------------------------------------
+template <typename Kern>
+cudaError_t grid_for(Kern kern, uint64_t n, int vecs_per_thread, const LaunchCfg& lc, unsigned* grid) {
+    int per_sm = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kBlock, 0);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const uint64_t tile = (uint64_t)kBlock * vecs_per_thread;
+    const uint64_t tiles = ((n >> 2) + tile - 1) / tile;
+    uint64_t g = (uint64_t)lc.sm_count * per_sm;
+    if (tiles < g) g = tiles;
+    if (g < 1) g = 1;
+    *grid = (unsigned)g;
+    return cudaSuccess;
+}
+
+constexpr int arrive_vecs(int K) { return K <= 1 ? 4 : (K <= 2 ? 2 : 1); }
+
+template <int K, bool DIAG, bool CUR>
+cudaError_t launch_arrive_k(const ArriveArgs& a, const LaunchCfg& lc, cudaStream_t s) {
+    constexpr int V = arrive_vecs(K);
+    auto kern = arrive_kernel<K, V, DIAG, CUR>;
+    unsigned grid = 1;
+    cudaError_t e = grid_for(kern, a.n, V, lc, &grid);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kBlock, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
+template <bool DIAG, bool CUR>
+cudaError_t launch_arrive_dc(const ArriveArgs& a, const LaunchCfg& lc, cudaStream_t s) {
+    switch (a.n_arr) {
+        case 0: return launch_arrive_k<0, false, false>(a, lc, s);
+        case 1: return launch_arrive_k<1, DIAG, CUR>(a, lc, s);
+        case 2: return launch_arrive_k<2, DIAG, CUR>(a, lc, s);
+        case 3: return launch_arrive_k<3, DIAG, CUR>(a, lc, s);
+        case 4: return launch_arrive_k<4, DIAG, CUR>(a, lc, s);
+        case 5: return launch_arrive_k<5, DIAG, CUR>(a, lc, s);
+        case 6: return launch_arrive_k<6, DIAG, CUR>(a, lc, s);
+        case 7: return launch_arrive_k<7, DIAG, CUR>(a, lc, s);
+        case 8: return launch_arrive_k<8, DIAG, CUR>(a, lc, s);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, const LaunchCfg& lc, cudaStream_t s) {
+    if (a.n == 0) return cudaSuccess;
+    if (a.n_arr > (uint32_t)kMaxArrivals || a.n_seed > (uint32_t)kMaxSeeds) return cudaErrorInvalidValue;
+    if (diagnostics) return pg_current ? launch_arrive_dc<true, true>(a, lc, s) : launch_arrive_dc<true, false>(a, lc, s);
+    return pg_current ? launch_arrive_dc<false, true>(a, lc, s) : launch_arrive_dc<false, false>(a, lc, s);
+}
+
+cudaError_t launch_adamw(const AdamArgs& a, const LaunchCfg& lc, cudaStream_t s) {
+    if (a.n == 0) return cudaSuccess;
+    constexpr int V = 2;
+    auto kern = adamw_kernel<V>;
+    unsigned grid = 1;
+    cudaError_t e = grid_for(kern, a.n, V, lc, &grid);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kBlock, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace alsgd
