@@ -1,0 +1,494 @@
+// Host side of the C ABI: flat-buffer layout, arena carving, Algorithm 3's counter and boundary
+// bookkeeping, worker dispatch state, and the translation of one ABI call into kernel launches.
+#include "../../include/alsgd.h"
+#include "alsgd_kernels.cuh"
+
+#include <cmath>
+#include <cstring>
+#include <limits>
+#include <new>
+#include <vector>
+
+using namespace alsgd;
+
+namespace {
+
+constexpr uint64_t kSliceAlign = 256;  // bytes; every arena slice starts on this boundary
+
+enum WorkerState : uint8_t { kNever = 0, kDispatched = 1, kArrived = 2 };
+
+struct Worker {
+    float* p = nullptr;
+    float* base = nullptr;
+    float* am = nullptr;
+    float* av = nullptr;
+    uint16_t* rep = nullptr;
+    uint64_t pull_tick = 0;
+    WorkerState state = kNever;
+};
+
+uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+    uint8_t* basep;
+    uint64_t off = 0;
+    explicit Carver(void* b) : basep(static_cast<uint8_t*>(b)) {}
+    template <typename T>
+    T* take(uint64_t count) {
+        off = round_up(off, kSliceAlign);
+        T* r = basep ? reinterpret_cast<T*>(basep + off) : nullptr;
+        off += count * sizeof(T);
+        return r;
+    }
+};
+
+struct Segments {
+    std::vector<uint64_t> end;
+    std::vector<uint32_t> decay;
+};
+
+// Flat offsets, padded total and the weight-decay segments of the flat vector: maximal runs of
+// elements with the same flag; padding between tensors is never decayed.
+bool build_layout(const alsgd_tensor_desc* t, uint32_t n, uint32_t align, uint64_t* P, uint64_t* offs, Segments* seg) {
+    if (!t || n == 0 || align == 0) return false;
+    const uint64_t lim = std::numeric_limits<uint64_t>::max() / 8;
+    uint64_t cur = 0;
+    auto push = [&](uint64_t end, uint32_t dec) {
+        if (!seg) return;
+        if (!seg->end.empty() && seg->decay.back() == dec) { seg->end.back() = end; return; }
+        seg->end.push_back(end);
+        seg->decay.push_back(dec);
+    };
+    for (uint32_t i = 0; i < n; ++i) {
+        if (t[i].numel == 0 || t[i].numel > lim || cur > lim) return false;
+        if (offs) offs[i] = cur;
+        const uint64_t end = cur + t[i].numel;
+        push(end, (t[i].flags & ALSGD_TENSOR_DECAY) ? 1u : 0u);
+        cur = round_up(end, align);
+        if (cur != end) push(cur, 0u);
+    }
+    if (cur > lim) return false;
+    *P = cur;
+    return true;
+}
+
+bool valid_cfg(const alsgd_config* c) {
+    if (!c) return false;
+    if (c->n_workers == 0 || c->N == 0) return false;
+    if (c->pg_base != ALSGD_PG_DISPATCH && c->pg_base != ALSGD_PG_CURRENT) return false;
+    if (c->flags & ~(ALSGD_CFG_REPLICA_BF16 | ALSGD_CFG_GRAD_STAGING)) return false;
+    if (!(c->beta >= 0.0f && c->beta < 1.0f)) return false;
+    if (!std::isfinite(c->outer_lr)) return false;
+    if (!(c->c >= 0.0f && (double)c->c * (double)c->N <= 1.0 + 1e-6)) return false;
+    if (!(c->adam_b1 >= 0.0f && c->adam_b1 < 1.0f && c->adam_b2 >= 0.0f && c->adam_b2 < 1.0f)) return false;
+    if (!(c->adam_eps >= 0.0f) || !(c->adam_wd >= 0.0f)) return false;
+    return true;
+}
+
+}  // namespace
+
+struct alsgd_ctx {
+    alsgd_config cfg;
+    uint64_t P = 0;
+    cudaStream_t stream = nullptr;
+    LaunchCfg lc{};
+    // device slices
+    uint64_t* seg_end = nullptr;
+    uint32_t* seg_decay = nullptr;
+    uint32_t n_seg = 0;
+    double* gnorm2 = nullptr;
+    unsigned int* nonfinite = nullptr;
+    float* theta = nullptr;
+    float* mom = nullptr;
+    float* delta = nullptr;
+    float* grad_stage = nullptr;
+    std::vector<Worker> workers;
+    // Algorithm 3 bookkeeping
+    uint64_t t = 0;
+    bool delta_zero = true;     // Delta is zero by definition (start, or right after a boundary)
+    bool delta_stored = true;   // ... and the arena really holds those zeros
+    // scalars of Algorithm 3, each rounded to fp32 once
+    float inv_n = 0, cb = 0, cn = 0;
+    int last_cuda = 0;
+};
+
+namespace {
+
+// Carve the arena; with arena == nullptr only the size is computed.
+uint64_t carve(alsgd_ctx* c, void* arena, uint64_t P, const alsgd_config& cfg, uint32_t n_seg) {
+    Carver k(arena);
+    uint64_t* seg_end = k.take<uint64_t>(n_seg);
+    uint32_t* seg_decay = k.take<uint32_t>(n_seg);
+    double* gn = k.take<double>(kMaxArrivals);
+    unsigned int* nf = k.take<unsigned int>(kMaxArrivals);
+    float* theta = k.take<float>(P);
+    float* mom = k.take<float>(P);
+    float* delta = k.take<float>(P);
+    if (c) {
+        c->seg_end = seg_end; c->seg_decay = seg_decay; c->gnorm2 = gn; c->nonfinite = nf;
+        c->theta = theta; c->mom = mom; c->delta = delta;
+        c->workers.assign(cfg.n_workers, Worker());
+    }
+    for (uint32_t w = 0; w < cfg.n_workers; ++w) {
+        float* p = k.take<float>(P);
+        float* base = cfg.pg_base == ALSGD_PG_DISPATCH ? k.take<float>(P) : nullptr;
+        float* am = k.take<float>(P);
+        float* av = k.take<float>(P);
+        uint16_t* rep = (cfg.flags & ALSGD_CFG_REPLICA_BF16) ? k.take<uint16_t>(P) : nullptr;
+        if (c) {
+            Worker& W = c->workers[w];
+            W.p = p; W.base = base; W.am = am; W.av = av; W.rep = rep;
+        }
+    }
+    float* stage = (cfg.flags & ALSGD_CFG_GRAD_STAGING) ? k.take<float>(P) : nullptr;
+    if (c) c->grad_stage = stage;
+    return round_up(k.off, kSliceAlign);
+}
+
+int cuda_fail(alsgd_ctx* c, cudaError_t e) {
+    if (c) c->last_cuda = (int)e;
+    return ALSGD_E_CUDA;
+}
+
+#define ALSGD_CUDA(ctx, call)                                   \
+    do {                                                        \
+        cudaError_t e__ = (call);                               \
+        if (e__ != cudaSuccess) return cuda_fail((ctx), e__);   \
+    } while (0)
+
+// Makes the context's device current for the duration of one ABI call.
+struct DeviceGuard {
+    int prev = -1;
+    int target = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) : target(dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() {
+        if (ok && prev >= 0 && prev != target) cudaSetDevice(prev);
+    }
+};
+
+int copy_vec(alsgd_ctx* c, void* dst, const void* src, uint64_t bytes, bool host_side) {
+    ALSGD_CUDA(c, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, c->stream));
+    if (host_side) ALSGD_CUDA(c, cudaStreamSynchronize(c->stream));
+    return ALSGD_OK;
+}
+
+void fill_seed(ArriveArgs& a, uint32_t slot, const Worker& w) {
+    a.seed_p[slot] = w.p;
+    a.seed_base[slot] = w.base;
+    a.seed_rep[slot] = w.rep;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* alsgd_strerror(int status) {
+    switch (status) {
+        case ALSGD_OK: return "ok";
+        case ALSGD_E_ARG: return "invalid argument";
+        case ALSGD_E_RANGE: return "index out of range";
+        case ALSGD_E_STATE: return "call not allowed in this state";
+        case ALSGD_E_CUDA: return "CUDA runtime error";
+        case ALSGD_E_NOMEM: return "not enough memory";
+        case ALSGD_E_UNSUPPORTED: return "unsupported";
+        default: return "unknown status";
+    }
+}
+
+int alsgd_layout_size(const alsgd_tensor_desc* tensors, uint32_t n, uint32_t align_elems,
+                      uint64_t* P_out, uint64_t* offsets_out) {
+    if (!P_out) return ALSGD_E_ARG;
+    uint64_t P = 0;
+    if (!build_layout(tensors, n, align_elems, &P, offsets_out, nullptr)) return ALSGD_E_ARG;
+    *P_out = P;
+    return ALSGD_OK;
+}
+
+int alsgd_arena_bytes(const alsgd_tensor_desc* tensors, uint32_t n, uint32_t align_elems,
+                      const alsgd_config* cfg, uint64_t* bytes_out) {
+    if (!bytes_out || !valid_cfg(cfg)) return ALSGD_E_ARG;
+    uint64_t P = 0;
+    Segments seg;
+    if (!build_layout(tensors, n, align_elems, &P, nullptr, &seg)) return ALSGD_E_ARG;
+    *bytes_out = carve(nullptr, nullptr, P, *cfg, (uint32_t)seg.end.size());
+    return ALSGD_OK;
+}
+
+int alsgd_init(alsgd_ctx** out, const alsgd_tensor_desc* tensors, uint32_t n, uint32_t align_elems,
+               const alsgd_config* cfg) {
+    if (!out || !valid_cfg(cfg) || !cfg->arena) return ALSGD_E_ARG;
+    if (reinterpret_cast<uintptr_t>(cfg->arena) % kSliceAlign) return ALSGD_E_ARG;
+    uint64_t P = 0;
+    Segments seg;
+    if (!build_layout(tensors, n, align_elems, &P, nullptr, &seg)) return ALSGD_E_ARG;
+    const uint64_t need = carve(nullptr, nullptr, P, *cfg, (uint32_t)seg.end.size());
+    if (cfg->arena_bytes < need) return ALSGD_E_NOMEM;
+
+    alsgd_ctx* c = new (std::nothrow) alsgd_ctx();
+    if (!c) return ALSGD_E_NOMEM;
+    c->cfg = *cfg;
+    c->P = P;
+    c->stream = static_cast<cudaStream_t>(cfg->stream);
+    c->n_seg = (uint32_t)seg.end.size();
+    carve(c, cfg->arena, P, *cfg, c->n_seg);
+    // Scalars of Algorithm 3: evaluated in double from the fp32 inputs, rounded to fp32 once.
+    c->inv_n = 1.0f / (float)cfg->N;
+    c->cb = (float)(((double)1.0 - (double)cfg->c * (double)cfg->N + (double)cfg->c) * (double)cfg->beta);
+    c->cn = (float)((double)cfg->c * (double)cfg->beta);
+
+    int rc = ALSGD_OK;
+    {
+        DeviceGuard g(cfg->device);
+        cudaError_t e = g.ok ? cudaSuccess : cudaErrorInvalidDevice;
+        int sms = 0;
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device);
+        c->lc.sm_count = sms;
+        if (e == cudaSuccess) e = cudaMemcpyAsync(c->seg_end, seg.end.data(), sizeof(uint64_t) * c->n_seg, cudaMemcpyHostToDevice, c->stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(c->seg_decay, seg.decay.data(), sizeof(uint32_t) * c->n_seg, cudaMemcpyHostToDevice, c->stream);
+        // The segment tables live in pageable host vectors that die with this scope.
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->gnorm2, 0, sizeof(double) * kMaxArrivals, c->stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * kMaxArrivals, c->stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->theta, 0, sizeof(float) * P, c->stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->mom, 0, sizeof(float) * P, c->stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->delta, 0, sizeof(float) * P, c->stream);
+        for (Worker& w : c->workers) {
+            if (e == cudaSuccess) e = cudaMemsetAsync(w.p, 0, sizeof(float) * P, c->stream);
+            if (e == cudaSuccess && w.base) e = cudaMemsetAsync(w.base, 0, sizeof(float) * P, c->stream);
+            if (e == cudaSuccess) e = cudaMemsetAsync(w.am, 0, sizeof(float) * P, c->stream);
+            if (e == cudaSuccess) e = cudaMemsetAsync(w.av, 0, sizeof(float) * P, c->stream);
+            if (e == cudaSuccess && w.rep) e = cudaMemsetAsync(w.rep, 0, sizeof(uint16_t) * P, c->stream);
+        }
+        if (e != cudaSuccess) { c->last_cuda = (int)e; rc = ALSGD_E_CUDA; }
+    }
+    if (rc != ALSGD_OK) { delete c; return rc; }
+    *out = c;
+    return ALSGD_OK;
+}
+
+int alsgd_destroy(alsgd_ctx* ctx) {
+    delete ctx;
+    return ALSGD_OK;
+}
+
+int alsgd_set_global(alsgd_ctx* c, const float* src, int src_is_device) {
+    if (!c || !src) return ALSGD_E_ARG;
+    DeviceGuard g(c->cfg.device);
+    return copy_vec(c, c->theta, src, sizeof(float) * c->P, !src_is_device);
+}
+
+int alsgd_get_global(alsgd_ctx* c, float* dst, int dst_is_device) {
+    if (!c || !dst) return ALSGD_E_ARG;
+    DeviceGuard g(c->cfg.device);
+    return copy_vec(c, dst, c->theta, sizeof(float) * c->P, !dst_is_device);
+}
+
+int alsgd_set_worker_params(alsgd_ctx* c, uint32_t worker, const float* src, int src_is_device) {
+    if (!c || !src) return ALSGD_E_ARG;
+    if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
+    DeviceGuard g(c->cfg.device);
+    return copy_vec(c, c->workers[worker].p, src, sizeof(float) * c->P, !src_is_device);
+}
+
+int alsgd_get_worker_params(alsgd_ctx* c, uint32_t worker, float* dst, int dst_is_device) {
+    if (!c || !dst) return ALSGD_E_ARG;
+    if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
+    DeviceGuard g(c->cfg.device);
+    return copy_vec(c, dst, c->workers[worker].p, sizeof(float) * c->P, !dst_is_device);
+}
+
+int alsgd_pull(alsgd_ctx* c, uint32_t worker) {
+    if (!c) return ALSGD_E_ARG;
+    if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
+    Worker& w = c->workers[worker];
+    ArriveArgs a{};
+    a.theta = c->theta;
+    a.n = c->P;
+    a.n_arr = 0;
+    a.n_seed = 1;
+    fill_seed(a, 0, w);
+    DeviceGuard g(c->cfg.device);
+    ALSGD_CUDA(c, launch_arrive(a, false, false, c->lc, c->stream));
+    w.pull_tick = c->t;
+    w.state = kDispatched;
+    return ALSGD_OK;
+}
+
+int alsgd_inner_adamw(alsgd_ctx* c, uint32_t worker, const float* grads, int grads_is_device,
+                      uint64_t step, float lr) {
+    if (!c || !grads || step == 0) return ALSGD_E_ARG;
+    if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
+    Worker& w = c->workers[worker];
+    if (w.state == kNever) return ALSGD_E_STATE;
+    if (!grads_is_device && !c->grad_stage) return ALSGD_E_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(grads) % 16) return ALSGD_E_ARG;
+    DeviceGuard g(c->cfg.device);
+    const float* gdev = grads;
+    if (!grads_is_device) {
+        ALSGD_CUDA(c, cudaMemcpyAsync(c->grad_stage, grads, sizeof(float) * c->P, cudaMemcpyHostToDevice, c->stream));
+        gdev = c->grad_stage;
+    }
+    AdamArgs a{};
+    a.p = w.p; a.m = w.am; a.v = w.av; a.g = gdev; a.rep = w.rep;
+    a.seg_end = c->seg_end; a.seg_decay = c->seg_decay; a.n_seg = c->n_seg;
+    a.n = c->P;
+    a.b1 = c->cfg.adam_b1; a.b2 = c->cfg.adam_b2;
+    a.omb1 = 1.0f - a.b1; a.omb2 = 1.0f - a.b2;
+    // Bias corrections: 1 - beta^step in double, rounded to fp32 once.
+    a.bc1 = (float)(1.0 - std::pow((double)a.b1, (double)step));
+    a.bc2 = (float)(1.0 - std::pow((double)a.b2, (double)step));
+    a.eps = c->cfg.adam_eps; a.lr = lr; a.wd = c->cfg.adam_wd;
+    ALSGD_CUDA(c, launch_adamw(a, c->lc, c->stream));
+    return ALSGD_OK;
+}
+
+int alsgd_arrive(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, alsgd_arrival_info* info) {
+    if (!c) return ALSGD_E_ARG;
+    if (flags & ~(ALSGD_ARRIVE_RESEED | ALSGD_ARRIVE_NORM | ALSGD_ARRIVE_NANCHECK)) return ALSGD_E_ARG;
+    if (k == 0) return ALSGD_OK;
+    if (!ids) return ALSGD_E_ARG;
+    const uint32_t W = c->cfg.n_workers;
+    if (k > W) return ALSGD_E_ARG;
+    std::vector<uint8_t> seen(W, 0);
+    for (uint32_t j = 0; j < k; ++j) {
+        if (ids[j] >= W) return ALSGD_E_RANGE;
+        if (seen[ids[j]]) return ALSGD_E_ARG;
+        seen[ids[j]] = 1;
+    }
+    for (uint32_t j = 0; j < k; ++j)
+        if (c->workers[ids[j]].state != kDispatched) return ALSGD_E_STATE;
+
+    const bool diag = (flags & (ALSGD_ARRIVE_NORM | ALSGD_ARRIVE_NANCHECK)) != 0;
+    const bool reseed = (flags & ALSGD_ARRIVE_RESEED) != 0;
+    const bool current = c->cfg.pg_base == ALSGD_PG_CURRENT;
+    const uint32_t N = c->cfg.N;
+    DeviceGuard g(c->cfg.device);
+
+    // Everything below only enqueues; the bookkeeping is committed after the last launch succeeded.
+    uint64_t t = c->t;
+    bool delta_zero = c->delta_zero, delta_stored = c->delta_stored;
+    std::vector<double> norms(k, 0.0);
+    std::vector<unsigned int> bads(k, 0u);
+
+    const uint32_t n_chunks = (k + kMaxArrivals - 1) / kMaxArrivals;
+    uint32_t seeded = 0;  // how many of the last ids[] the final arrival launch re-seeds itself
+    for (uint32_t ch = 0; ch < n_chunks; ++ch) {
+        const uint32_t j0 = ch * kMaxArrivals;
+        const uint32_t kk = (k - j0 < (uint32_t)kMaxArrivals) ? k - j0 : (uint32_t)kMaxArrivals;
+        ArriveArgs a{};
+        a.theta = c->theta; a.delta = c->delta; a.mom = c->mom;
+        a.gnorm2 = c->gnorm2; a.nonfinite = c->nonfinite;
+        a.n = c->P;
+        a.n_arr = kk;
+        a.beta = c->cfg.beta; a.eps = c->cfg.outer_lr; a.inv_n = c->inv_n; a.cb = c->cb; a.cn = c->cn;
+        bool any_boundary = false, last_boundary = false;
+        for (uint32_t j = 0; j < kk; ++j) {
+            const Worker& w = c->workers[ids[j0 + j]];
+            a.p[j] = w.p;
+            a.base[j] = w.base;
+            const bool b = ((t + j + 1) % N) == 0;          // Algorithm 3's boundary test
+            if (b) { a.boundary_mask |= 1u << j; any_boundary = true; }
+            last_boundary = b;
+        }
+        if (delta_zero) a.flags |= kDeltaZeroIn;
+        if (last_boundary) a.flags |= kDeltaSkipStore;
+        if (c->cfg.c != 0.0f) a.flags |= kCNonZero | kReadM;
+        if (any_boundary) a.flags |= kReadM | kWriteM;
+        if (reseed && ch + 1 == n_chunks) {               // the final theta exists only in the last pass
+            const uint32_t ns = k < (uint32_t)kMaxSeeds ? k : (uint32_t)kMaxSeeds;
+            for (uint32_t s = 0; s < ns; ++s) fill_seed(a, s, c->workers[ids[k - ns + s]]);
+            a.n_seed = ns;
+            seeded = ns;
+        }
+        if (diag) {
+            ALSGD_CUDA(c, cudaMemsetAsync(c->gnorm2, 0, sizeof(double) * kMaxArrivals, c->stream));
+            ALSGD_CUDA(c, cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * kMaxArrivals, c->stream));
+        }
+        ALSGD_CUDA(c, launch_arrive(a, current, diag, c->lc, c->stream));
+        if (diag && info) {
+            ALSGD_CUDA(c, cudaMemcpyAsync(norms.data() + j0, c->gnorm2, sizeof(double) * kk, cudaMemcpyDeviceToHost, c->stream));
+            ALSGD_CUDA(c, cudaMemcpyAsync(bads.data() + j0, c->nonfinite, sizeof(unsigned int) * kk, cudaMemcpyDeviceToHost, c->stream));
+            ALSGD_CUDA(c, cudaStreamSynchronize(c->stream));
+        }
+        t += kk;
+        delta_zero = last_boundary;
+        delta_stored = !last_boundary;
+    }
+    // A batch larger than one launch can re-seed: the remaining workers get the same final theta.
+    if (reseed && seeded < k) {
+        uint32_t left = k - seeded, at = 0;
+        while (left) {
+            const uint32_t ns = left < (uint32_t)kMaxSeeds ? left : (uint32_t)kMaxSeeds;
+            ArriveArgs a{};
+            a.theta = c->theta; a.n = c->P; a.n_seed = ns;
+            for (uint32_t s = 0; s < ns; ++s) fill_seed(a, s, c->workers[ids[at + s]]);
+            ALSGD_CUDA(c, launch_arrive(a, false, false, c->lc, c->stream));
+            at += ns; left -= ns;
+        }
+    }
+
+    // ---- commit bookkeeping
+    if (info) {
+        for (uint32_t j = 0; j < k; ++j) {
+            alsgd_arrival_info& o = info[j];
+            o.tick = c->t + j;
+            o.staleness = o.tick - c->workers[ids[j]].pull_tick;
+            o.worker = ids[j];
+            o.boundary = ((c->t + j + 1) % N) == 0 ? 1u : 0u;
+            o.gnorm2 = (flags & ALSGD_ARRIVE_NORM) ? norms[j] : 0.0;
+            o.nonfinite = (flags & ALSGD_ARRIVE_NANCHECK) ? (bads[j] ? 1u : 0u) : 0u;
+            o.reserved = 0;
+        }
+    }
+    c->t = t;
+    c->delta_zero = delta_zero;
+    c->delta_stored = delta_stored;
+    for (uint32_t j = 0; j < k; ++j) {
+        Worker& w = c->workers[ids[j]];
+        if (reseed) { w.state = kDispatched; w.pull_tick = c->t; }
+        else w.state = kArrived;
+    }
+    return ALSGD_OK;
+}
+
+int alsgd_counters(alsgd_ctx* c, uint64_t* t_out, uint32_t* phase_out) {
+    if (!c) return ALSGD_E_ARG;
+    if (t_out) *t_out = c->t;
+    if (phase_out) *phase_out = (uint32_t)(c->t % c->cfg.N);
+    return ALSGD_OK;
+}
+
+int alsgd_state_ptrs(alsgd_ctx* c, alsgd_ptrs* out) {
+    if (!c || !out) return ALSGD_E_ARG;
+    if (c->delta_zero && !c->delta_stored) {
+        DeviceGuard g(c->cfg.device);
+        ALSGD_CUDA(c, cudaMemsetAsync(c->delta, 0, sizeof(float) * c->P, c->stream));
+        c->delta_stored = true;
+    }
+    out->theta = c->theta; out->m = c->mom; out->delta = c->delta;
+    out->P = c->P; out->n_workers = c->cfg.n_workers; out->reserved = 0;
+    return ALSGD_OK;
+}
+
+int alsgd_worker_state_ptrs(alsgd_ctx* c, uint32_t worker, alsgd_worker_ptrs* out) {
+    if (!c || !out) return ALSGD_E_ARG;
+    if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
+    const Worker& w = c->workers[worker];
+    out->p = w.p; out->base = w.base; out->adam_m = w.am; out->adam_v = w.av; out->replica = w.rep;
+    return ALSGD_OK;
+}
+
+int alsgd_sync(alsgd_ctx* c) {
+    if (!c) return ALSGD_E_ARG;
+    DeviceGuard g(c->cfg.device);
+    ALSGD_CUDA(c, cudaStreamSynchronize(c->stream));
+    return ALSGD_OK;
+}
+
+int alsgd_last_cuda_error(alsgd_ctx* c) { return c ? c->last_cuda : 0; }
+
+}  // extern "C"
