@@ -1,0 +1,358 @@
+"""Benchmark of the asynchronous Local-SGD server path on B200.
+
+One step = one arrival of the seeded heterogeneous schedule on the ~110M-parameter layout: the host
+scheduler (Algorithm 2/5) names the arriving worker, that worker runs its DyLU number of inner AdamW
+steps (Eq. 6; 16/25/33/50 for speeds 1:1.5:2:3, H = 50), then its pseudo-gradient goes through the
+Delayed-Nesterov arrival with the fused re-seed.  Each kernel launch streams the whole flat vector
+(3.3-3.7 GB per launch, far larger than L2), so no L2 flush is needed between iterations.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line on rank 0.
+"""
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "params_per_s_dn_arrival_plus_adamw"
+UNIT = "params/s"
+WORKLOAD = "decoder-110M(12L,d768,ff3072,V32000) W=4 N=4 beta=0.9 outer_lr=0.7 c=0 bf16-replicas"
+SPEEDS = [1.0, 1.5, 2.0, 3.0]
+H = 50
+ADAMW_BYTES = 30          # g,p,m,v read (16) + p,m,v write (12) + bf16 replica write (2)
+ARRIVE_RESEED_BYTES = {   # theta, Delta, base, p read / theta, Delta write (+m on a boundary), + p, base, bf16 re-seed
+    "first": 20 + 10,     # Delta known zero: not read
+    "middle": 24 + 10,
+    "boundary": 28 + 10,  # + m read and write; Delta zero store elided
+}
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per parameter from the committed ncu captures
+# (profiles/), valid only for the kernel source they were taken from.
+NCU_TRAFFIC = {
+    "src_sha256": None,
+    "adamw_bytes_per_param": None,
+    "arrive_bytes_per_param": None,
+}
+
+
+def kernel_source_hash():
+    h = hashlib.sha256()
+    with open(os.path.join(ROOT, "paper_2401_09135_b200", "csrc", "alsgd_kernels.cu"), "rb") as f:
+        h.update(f.read())
+    return h.hexdigest()
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled while the timed region runs (read-only)."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.rows:
+            if not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            f = [x.strip() for x in line.split(",")]
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_schedule(n_arrivals):
+    """Arrival order from the library's host scheduler, DyLU steps from Eq. 6."""
+    from paper_2401_09135_b200 import binding as B, synth
+    steps = B.alsgd_dylu_steps(SPEEDS, H)
+    dur = synth.job_durations(SPEEDS, steps, n_arrivals + 2, synth.SEED + 7)
+    s = B.Scheduler(len(SPEEDS), 0.0)
+    rounds = [0] * len(SPEEDS)
+    for w in range(len(SPEEDS)):
+        s.dispatch(w, dur[w, 0], steps[w])
+    order = []
+    while len(order) < n_arrivals:
+        ids, _, _ = s.next_batch()
+        for w in ids:
+            order.append(w)
+            rounds[w] += 1
+            s.dispatch(w, dur[w, rounds[w]], steps[w])
+    return steps, order[:n_arrivals]
+
+
+# ----------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+# ----------------------------------------------------------------------------------------------------
+def oracle_step(srv, w, n_inner, grads, life, lr=1e-3):
+    for _ in range(n_inner):
+        life[w] += 1
+        srv.inner_adamw(w, grads[life[w] % len(grads)], life[w], lr)
+    srv.arrive([w], reseed_after=True)
+
+
+def run_oracle(n_elems, order, steps, warmup, timed):
+    """Times `timed` steps of the same path on the first n_elems elements of the layout."""
+    import numpy as np
+    import oracle
+    from paper_2401_09135_b200 import synth
+    tensors = synth.layout_110m()
+    offs, P = oracle.layout_offsets([t.numel for t in tensors], 128)
+    mask = oracle.decay_mask([t.numel for t in tensors], [t.decay for t in tensors], offs, P)[:n_elems].copy()
+    srv = oracle.OracleServer(n_elems, len(SPEEDS), 4, 0.9, 0.7, decay=mask)
+    srv.set_global(synth.normal_vec(n_elems, 0.02, synth.SEED, synth.STREAM_THETA0))
+    grads = [synth.normal_vec(n_elems, 1e-2, synth.SEED, synth.STREAM_GRAD, sub=i) for i in range(2)]
+    for w in range(len(SPEEDS)):
+        srv.pull(w)
+    life = [0] * len(SPEEDS)
+    for w in order[:warmup]:
+        oracle_step(srv, w, steps[w], grads, life)
+    t0 = time.perf_counter()
+    passes = 0
+    for w in order[warmup:warmup + timed]:
+        oracle_step(srv, w, steps[w], grads, life)
+        passes += steps[w] + 1
+    dt = time.perf_counter() - t0
+    return n_elems * passes / dt, dt, passes
+
+
+def main_reference(args, rank):
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    steps, order = build_schedule(args.warmup + args.steps)
+    n_elems = 1 << 22
+    value, dt, passes = run_oracle(n_elems, order, steps, args.warmup, args.steps)
+    sample = f"first {n_elems} elements of the layout, every step of the schedule (DyLU inner steps + arrival)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "H": H, "speeds": SPEEDS, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------------------
+def main_ours(args, rank, world, local_rank):
+    import numpy as np
+    import torch
+    from paper_2401_09135_b200 import binding as B, synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    tensors = synth.layout_110m()
+    ctx = B.Context(tensors, len(SPEEDS), 4, 0.9, 0.7, grad_staging=True, device=local_rank)
+    P = ctx.P
+    n_total = args.warmup + args.steps
+    steps, order = build_schedule(2 * n_total)
+    theta0 = synth.theta0(tensors, ctx.offsets, P, synth.SEED + rank)
+    ctx.alsgd_set_global(theta0)
+    for w in range(len(SPEEDS)):
+        ctx.alsgd_pull(w)
+    G = 2
+    gpool_host = [torch.from_numpy(synth.normal_vec(P, 1e-2, synth.SEED + rank, synth.STREAM_GRAD, sub=i)).pin_memory()
+                  for i in range(G)]
+    gpool = [g.cuda(non_blocking=True) for g in gpool_host]
+    theta_host = torch.empty(P, dtype=torch.float32).pin_memory()
+    life = [0] * len(SPEEDS)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def run(seq, pool, host_io, timers=None):
+        """Runs the arrivals in seq; returns the number of kernel launches."""
+        launches = 0
+        for w in seq:
+            if timers is not None:
+                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                e0.record()
+            for _ in range(steps[w]):
+                life[w] += 1
+                ctx.alsgd_inner_adamw(w, pool[synth.grad_pool_index(w, life[w], G)], life[w], 1e-3)
+            if timers is not None:
+                e1.record()
+            ctx.alsgd_arrive([w], B.ARRIVE_RESEED, want_info=False)
+            if timers is not None:
+                e2.record()
+                timers.append((w, e0, e1, e2))
+            if host_io:
+                ctx.alsgd_get_global(theta_host)          # waits: the worker's next round needs the model
+            launches += steps[w] + 1
+        return launches
+
+    # ---- device-resident throughput
+    run(order[:args.warmup], gpool, False)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    t_wall0 = time.time()
+    start_evt, stop_evt = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    timers = []
+    start_evt.record()
+    launches = run(order[args.warmup:n_total], gpool, False, timers)
+    stop_evt.record()
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    ms = start_evt.elapsed_time(stop_evt)
+    passes = launches
+    adam_ms = sum(e0.elapsed_time(e1) for _, e0, e1, _ in timers)
+    adam_launches = sum(steps[w] for w, *_ in timers)
+    arr_ms = sum(e1.elapsed_time(e2) for _, _, e1, e2 in timers)
+    arr_launches = len(timers)
+
+    # ---- end to end: gradients come from pinned host memory every inner step, theta goes back each arrival
+    e2e_seq = order[n_total:n_total + args.steps]
+    run(e2e_seq[:1], gpool_host, True)
+    barrier()
+    s2, t2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    e2e_launches = run(e2e_seq, gpool_host, True)
+    t2.record()
+    barrier()
+    e2e_ms = s2.elapsed_time(t2)
+    h2d = sum(steps[w] for w in e2e_seq) * 4 * P / len(e2e_seq)
+    d2h = 4 * P
+
+    times = torch.tensor([ms, e2e_ms, adam_ms / adam_launches, arr_ms / arr_launches], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms, e2e_ms, adam_avg_ms, arr_avg_ms = [float(x) for x in times.cpu()]
+
+    if rank == 0:
+        peak, which = measured_peak()
+        value = world * P * passes / (ms * 1e-3)
+        e2e_value = world * P * e2e_launches / (e2e_ms * 1e-3)
+        adam_gbs = ADAMW_BYTES * P / (adam_avg_ms * 1e-3) / 1e9
+        # arrival bytes: by Delayed-Nesterov phase of each timed arrival (N = 4; the warm-up took ticks 0..warmup-1)
+        kinds = ["first" if (args.warmup + i) % 4 == 0 else "boundary" if (args.warmup + i) % 4 == 3 else "middle"
+                 for i in range(arr_launches)]
+        arr_bytes = sum(ARRIVE_RESEED_BYTES[k] for k in kinds) / float(arr_launches)
+        arr_gbs = arr_bytes * P / (arr_avg_ms * 1e-3) / 1e9
+        traffic_ok = NCU_TRAFFIC["src_sha256"] == kernel_source_hash()
+        adam_traffic = NCU_TRAFFIC["adamw_bytes_per_param"] * P if traffic_ok and NCU_TRAFFIC["adamw_bytes_per_param"] else None
+        arr_traffic = NCU_TRAFFIC["arrive_bytes_per_param"] * P if traffic_ok and NCU_TRAFFIC["arrive_bytes_per_param"] else None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "P": P, "H": H, "speeds": SPEEDS, "dylu_steps": steps,
+                       "step": "one scheduled arrival: DyLU inner AdamW steps of the arriving worker + DN arrival with fused re-seed",
+                       "l2": "every launch streams 3.3-3.7 GB (inputs larger than the 126 MB L2); no flush needed",
+                       "multi_gpu": "each rank holds its own 110M-element range of an N-times larger vector; no exchange"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms / len(e2e_seq)},
+            "gpu_launches": launches,
+            "roofline": {"kernel": "adamw_kernel (fused AdamW + bf16 cast)", "bound": "hbm", "achieved": adam_gbs,
+                         "peak": peak, "peak_source": f"of {which}", "unit": "GB/s", "frac": adam_gbs / peak,
+                         "frac_of_nominal_8TBs": adam_gbs / NOMINAL_HBM_GBS, "traffic": adam_traffic,
+                         "bytes_per_param": ADAMW_BYTES, "launches": adam_launches, "avg_ms": adam_avg_ms},
+            "roofline_arrive": {"kernel": "arrive_kernel<K=1> (pseudo-gradient + Delayed Nesterov + re-seed)", "bound": "hbm",
+                                "achieved": arr_gbs, "peak": peak, "peak_source": f"of {which}", "unit": "GB/s",
+                                "frac": arr_gbs / peak, "frac_of_nominal_8TBs": arr_gbs / NOMINAL_HBM_GBS,
+                                "traffic": arr_traffic, "bytes_per_param": arr_bytes, "launches": arr_launches,
+                                "avg_ms": arr_avg_ms},
+            "params_per_s": {"adamw": P / (adam_avg_ms * 1e-3), "dn_arrival_reseed": P / (arr_avg_ms * 1e-3)},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            n_cpu = P // 8
+            cpu_order = [order[0]]
+            v, dt, p = run_oracle(n_cpu, cpu_order, steps, 0, 1)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
+                                    "sample": f"first {n_cpu} elements (an eighth) of the layout, one step: {steps[cpu_order[0]]} inner AdamW steps + 1 arrival with re-seed"}
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        main_reference(args, rank)
+    else:
+        main_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
