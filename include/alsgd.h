@@ -236,6 +236,35 @@ int alsgd_sched_next_batch(alsgd_sched* s, uint32_t* ids_out, double* times_out,
 /* Total local updates synchronised so far (Algorithm 2's t_local). */
 int alsgd_sched_local_updates(alsgd_sched* s, uint64_t* t_local_out);
 
+/* ------------------------------------------------------------------------------------------------
+ * Diagnostics without any allocation (the paper has no counterpart; this serves embedders)
+ * ---------------------------------------------------------------------------------------------- */
+
+/* Largest vector alsgd_pg_norm_static accepts. */
+#define ALSGD_STATIC_MAX_ELEMS (1ull << 27)
+
+/* Squared norm and non-finite flag of a pseudo-gradient start - p, for callers that cannot obtain
+ * device memory of their own: code hosted inside another framework's memory plan or between its
+ * graph launches, or a process whose device memory was all handed out at start-up.  It needs no
+ * context and no arena.  Its working memory (one flag word plus one double per 4096 elements,
+ * 256 KiB + 256 bytes in total) is a fixed array inside the library image, which every GPU that
+ * loads the library holds until the process exits; the call itself invokes no allocating routine.
+ *   start, p        device, n fp32 values each, 16-byte aligned, caller-owned (for a worker of a
+ *                   context: its dispatch snapshot and its parameters)
+ *   n               1 .. ALSGD_STATIC_MAX_ELEMS; more returns ALSGD_E_NOMEM and does nothing
+ *   device, stream  the device that owns the buffers and the stream to enqueue on
+ *   gnorm2_out      device, one double: sum of (start[i] - p[i])^2, accumulated in double in a fixed
+ *                   order (the same inputs give the same bits on every call)
+ *   nonfinite_out   device, one uint32: 1 if any entry of start - p is NaN or Inf, else 0
+ * The call only enqueues; the outputs are valid once the stream reaches them.  The first call on each
+ * device looks up the array's device address; make that first call outside any stream capture.
+ * All calls on one device share the one array and it keeps the previous call's contents, so the call
+ * clears what it accumulates into before use; two calls whose kernels can overlap on the GPU (other
+ * streams, other threads) race on it and must be ordered by the caller.
+ * ALSGD_E_ARG: null or misaligned pointer, n = 0.  ALSGD_E_RANGE: device ordinal outside 0..63. */
+int alsgd_pg_norm_static(const float* start, const float* p, uint64_t n, int32_t device, void* stream,
+                         double* gnorm2_out, uint32_t* nonfinite_out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -81,7 +81,9 @@ SIGNATURES = {
     "alsgd_sched_dispatch": (C.c_int, [_vp, C.c_uint32, C.c_double, C.c_uint32]),
     "alsgd_sched_next_batch": (C.c_int, [_vp, _u32p, _f64p, C.c_uint32, _u32p, _f64p]),
     "alsgd_sched_local_updates": (C.c_int, [_vp, _u64p]),
+    "alsgd_pg_norm_static": (C.c_int, [_vp, _vp, C.c_uint64, C.c_int32, _vp, _vp, _vp]),
 }
+STATIC_MAX_ELEMS = 1 << 27
 
 _lib = None
 

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libalsgd.so")
-SOURCES = ["alsgd_kernels.cu", "alsgd_ctx.cu", "alsgd_sched.cpp"]
+SOURCES = ["alsgd_kernels.cu", "alsgd_ctx.cu", "alsgd_sched.cpp", "alsgd_static.cu"]
 HEADERS = [os.path.join(CSRC, "alsgd_kernels.cuh"), os.path.join(HERE, "..", "include", "alsgd.h")]
 
 NVCC_FLAGS = [
