@@ -1,0 +1,43 @@
+"""A small fixed case for profiler captures: a few launches of each kernel on vectors larger than L2
+but only ~2.4 GB on the device in total.
+
+    python -m paper_2401_09135_b200.profile_case [--elems N]
+
+Launch order: 2 pulls, 3 AdamW steps on worker 0, 3 on worker 1, then single arrivals with fused
+re-seed through one Delayed-Nesterov cycle of N = 4 (first / middle / middle / boundary), then one
+batch of two.
+"""
+import argparse
+
+import torch
+
+from . import binding as B
+from . import synth
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--elems", type=int, default=48 * 1024 * 1024)
+    args = ap.parse_args()
+    n = args.elems
+    tensors = [synth.Tensor("w0", n // 2, True, "matrix"), synth.Tensor("g0", 4096, False, "gain"),
+               synth.Tensor("w1", n - n // 2 - 4096, True, "matrix")]
+    ctx = B.Context(tensors, 2, 4, 0.9, 0.7)
+    theta0 = torch.from_numpy(synth.theta0(tensors, ctx.offsets, ctx.P))
+    ctx.alsgd_set_global(theta0.numpy())
+    g = torch.from_numpy(synth.normal_vec(ctx.P, 1e-2, synth.SEED, synth.STREAM_GRAD)).cuda()
+    for w in range(2):
+        ctx.alsgd_pull(w)
+    for w in range(2):
+        for s in range(1, 4):
+            ctx.alsgd_inner_adamw(w, g, s, 1e-3)
+    for w in (0, 1, 0, 1):
+        ctx.alsgd_arrive([w], B.ARRIVE_RESEED, want_info=False)
+    ctx.alsgd_arrive([0, 1], B.ARRIVE_RESEED, want_info=False)
+    ctx.alsgd_sync()
+    print(f"profile case done: P={ctx.P}, t={ctx.alsgd_counters()[0]}")
+    ctx.close()
+
+
+if __name__ == "__main__":
+    main()
