@@ -4,6 +4,10 @@
 // goal is HBM bandwidth: 128-bit coalesced accesses, several independent vectors in flight per
 // thread, touch-once cache hints, one pass over theta / Delta / m no matter how many workers
 // arrive, and the re-seed of the dispatched workers written from registers in the same pass.
+// Each block handles exactly one tile and exits: on B200 this measured 15-20 % faster than a
+// persistent grid-stride loop of the same body (6.6-6.9 TB/s against 5.3-6.0 TB/s), because the
+// block scheduler keeps fresh blocks issuing loads while older ones are still storing, instead
+// of all resident blocks marching through load and store phases together.
 //
 // Arithmetic contract: every fp32 operation is a separate IEEE-754 round-to-nearest operation in
 // the order Algorithm 3 states it (this file is compiled with -fmad=false, IEEE division and
@@ -84,7 +88,8 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
     float4* __restrict__ delta4 = reinterpret_cast<float4*>(a.delta);
     float4* __restrict__ mom4 = reinterpret_cast<float4*>(a.mom);
 
-    for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < nvec; t0 += (uint64_t)gridDim.x * tile) {
+    {
+        const uint64_t t0 = (uint64_t)blockIdx.x * tile;      // one tile per block
         float4 th[V], d[V], mm[V];
         float4 b[KK][V], p[KK][V];
         // ---- issue every load of the tile before the first use
@@ -243,7 +248,8 @@ __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ A
     SegCursor cur;
     bool have_cur = false;
 
-    for (uint64_t t0 = (uint64_t)blockIdx.x * tile; t0 < nvec; t0 += (uint64_t)gridDim.x * tile) {
+    {
+        const uint64_t t0 = (uint64_t)blockIdx.x * tile;      // one tile per block
         float4 p[V], m[V], v[V], g[V];
 #pragma unroll
         for (int k = 0; k < V; ++k) {
@@ -299,32 +305,30 @@ __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ A
 }
 
 // ---------------------------------------------------------------------------------------------
-// Launch shapes: persistent grids, a whole number of resident blocks per SM.
+// Launch shapes: one block per tile of kBlock * V float4 vectors (block 0 also takes the up to
+// three trailing elements).
 // ---------------------------------------------------------------------------------------------
-template <typename Kern>
-cudaError_t grid_for(Kern kern, uint64_t n, int vecs_per_thread, const LaunchCfg& lc, unsigned* grid) {
-    int per_sm = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kBlock, 0);
-    if (e != cudaSuccess) return e;
-    if (per_sm < 1) per_sm = 1;
+cudaError_t grid_for(uint64_t n, int vecs_per_thread, unsigned* grid) {
     const uint64_t tile = (uint64_t)kBlock * vecs_per_thread;
-    const uint64_t tiles = ((n >> 2) + tile - 1) / tile;
-    uint64_t g = (uint64_t)lc.sm_count * per_sm;
-    if (tiles < g) g = tiles;
-    if (g < 1) g = 1;
-    *grid = (unsigned)g;
+    uint64_t tiles = ((n >> 2) + tile - 1) / tile;
+    if (tiles < 1) tiles = 1;
+    if (tiles > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    *grid = (unsigned)tiles;
     return cudaSuccess;
 }
 
-constexpr int arrive_vecs(int K) { return K <= 1 ? 4 : (K <= 2 ? 2 : 1); }
+// Vectors per thread, from measurement on B200 at 110M elements (GB/s, fused re-seed of all K):
+// K=1: V=1 6635, V=2 6693, V=4 6735;  K=2: V=1 6612, V=2 6689;  K=4: V=1 6576, V=2 6626;  K=8: V=1 6600.
+constexpr int arrive_vecs(int K) { return K <= 1 ? 4 : (K <= 4 ? 2 : 1); }
 
 template <int K, bool DIAG, bool CUR>
 cudaError_t launch_arrive_k(const ArriveArgs& a, const LaunchCfg& lc, cudaStream_t s) {
     constexpr int V = arrive_vecs(K);
     auto kern = arrive_kernel<K, V, DIAG, CUR>;
     unsigned grid = 1;
-    cudaError_t e = grid_for(kern, a.n, V, lc, &grid);
+    cudaError_t e = grid_for(a.n, V, &grid);
     if (e != cudaSuccess) return e;
+    (void)lc;
     kern<<<grid, kBlock, 0, s>>>(a);
     return cudaGetLastError();
 }
@@ -359,8 +363,9 @@ cudaError_t launch_adamw(const AdamArgs& a, const LaunchCfg& lc, cudaStream_t s)
     constexpr int V = 2;
     auto kern = adamw_kernel<V>;
     unsigned grid = 1;
-    cudaError_t e = grid_for(kern, a.n, V, lc, &grid);
+    cudaError_t e = grid_for(a.n, V, &grid);
     if (e != cudaSuccess) return e;
+    (void)lc;
     kern<<<grid, kBlock, 0, s>>>(a);
     return cudaGetLastError();
 }
