@@ -281,10 +281,9 @@ def main_ours(args, rank, world, local_rank):
     h2d = sum(steps[w] for w in e2e_seq) * 4 * P / len(e2e_seq)
     d2h = 4 * P
 
-    times = torch.tensor([ms, e2e_ms, adam_ms / adam_launches, arr_ms / arr_launches], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, e2e_ms, adam_avg_ms, arr_avg_ms = [float(x) for x in times.cpu()]
+    from paper_2401_09135_b200 import shard
+    ms, e2e_ms, adam_avg_ms, arr_avg_ms = shard.max_over_ranks(
+        [ms, e2e_ms, adam_ms / adam_launches, arr_ms / arr_launches], device="cuda")
 
     if rank == 0:
         peak, which = measured_peak()
@@ -337,6 +336,63 @@ def main_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def main_ksweep(args):
+    """Arrival-batch sweep on the 110M layout with 8 resident workers (N = 8): per k, each round is 8/k
+    batches of k through the multi-arrival kernel with fused re-seed, then 10 AdamW steps per worker."""
+    import torch
+    from paper_2401_09135_b200 import binding as B, synth
+    torch.cuda.set_device(0)
+    tensors = synth.layout_110m()
+    W, N, inner = 8, 8, 10
+    peak, which = measured_peak()
+    out = []
+    gpool = None
+    for k in (1, 2, 4, 8):
+        ctx = B.Context(tensors, W, N, 0.9, 0.7)
+        P = ctx.P
+        if gpool is None:
+            gpool = [torch.from_numpy(synth.normal_vec(P, 1e-2, synth.SEED, synth.STREAM_GRAD, sub=i)).cuda() for i in range(2)]
+        ctx.alsgd_set_global(synth.theta0(tensors, ctx.offsets, P))
+        for w in range(W):
+            ctx.alsgd_pull(w)
+        order = [int(w) for w in synth.rng(synth.SEED + 8, synth.STREAM_ORDER, k).permutation(W)]
+        life = [0] * W
+        rounds = args.warmup // 4 + 1 + max(5, args.steps // 3)
+        ev = []
+        for r in range(rounds):
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record()
+            for i in range(0, W, k):
+                ctx.alsgd_arrive(order[i:i + k], B.ARRIVE_RESEED, want_info=False)
+            e1.record()
+            for w in range(W):
+                for _ in range(inner):
+                    life[w] += 1
+                    ctx.alsgd_inner_adamw(w, gpool[synth.grad_pool_index(w, life[w], 2)], life[w], 1e-3)
+            e2.record()
+            ev.append((e0, e1, e2))
+        torch.cuda.synchronize()
+        ev = ev[1:]                                        # first round is warm-up
+        arr_ms = sum(a.elapsed_time(b) for a, b, _ in ev) / len(ev)
+        adam_ms = sum(b.elapsed_time(c) for _, b, c in ev) / len(ev)
+        # one full cycle per round (N = W = 8): Delta read on all batches but the first, written on all but
+        # the last, m read+written once; per arrival 8 B of (base, p) reads and 10 B of re-seed writes
+        nb = W // k
+        arr_bytes = (4 * nb + 4 * (nb - 1) + 4 * nb + 4 * (nb - 1) + 8 + 18 * W) * P
+        adam_bytes = ADAMW_BYTES * P * W * inner
+        out.append({"k": k, "arrival_ms_per_round": arr_ms, "arrival_gbs": arr_bytes / arr_ms / 1e6,
+                    "arrival_frac": arr_bytes / arr_ms / 1e6 / peak, "arrival_bytes_per_param_per_arrival": arr_bytes / P / W,
+                    "arrivals_per_s": W / (arr_ms * 1e-3), "adamw_ms_per_round": adam_ms,
+                    "adamw_gbs": adam_bytes / adam_ms / 1e6, "adamw_frac": adam_bytes / adam_ms / 1e6 / peak,
+                    "combined_gbs": (arr_bytes + adam_bytes) / (arr_ms + adam_ms) / 1e6,
+                    "combined_frac": (arr_bytes + adam_bytes) / (arr_ms + adam_ms) / 1e6 / peak})
+        ctx.close()
+        del ctx
+        torch.cuda.empty_cache()
+    print(json.dumps({"workload": "decoder-110M W=8 N=8 beta=0.9 outer_lr=0.7, k-sweep, 10 inner AdamW steps per worker per round",
+                      "peak_gbs": peak, "peak_source": f"of {which}", "unit": "GB/s", "rounds_timed": len(ev), "sweep": out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -344,11 +400,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ksweep", action="store_true", help="arrival-batch sweep (k = 1, 2, 4, 8) with 8 resident workers")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
+    if args.ksweep:
+        main_ksweep(args)
+    elif args.impl == "reference":
         main_reference(args, rank)
     else:
         main_ours(args, rank, world, local_rank)
