@@ -214,15 +214,27 @@ class OracleServer:
         b1, b2, eps, wd = self.adam
         adamw(self.p[w], self.am[w], self.av[w], grads, self.replica[w], self.decay, step, lr, b1, b2, eps, wd)
 
-    def arrive(self, ids, reseed_after=True, norm=False, weights=None, dc_lambda=0.0, buffered=False):
+    def arrive(self, ids, reseed_after=True, norm=False, weights=None, dc_lambda=0.0, buffered=False,
+               poly=False, stale_threshold=None):
         """Apply the arrivals of one grace window in the given order, then (optionally) re-dispatch
-        all of them with the final global model.  Returns one info dict per arrival."""
+        all of them with the final global model.  Returns one info dict per arrival.
+
+        poly: weight each pseudo-gradient by (1 + staleness)^-0.5 (Section 4, "Async. DiLoCo + Poly").
+        stale_threshold: with poly, discard updates whose staleness exceeds it ("PolyThres"); a
+        discarded update is not a server update (t does not advance) but its worker is re-dispatched."""
         infos = []
         for j, w in enumerate(ids):
-            info = {"worker": w, "tick": self.t, "staleness": self.t - self.pull_tick[w]}
+            stale = self.t - self.pull_tick[w]
+            info = {"worker": w, "tick": self.t, "staleness": stale, "dropped": False, "boundary": False}
             if norm:
                 info["gnorm2"], info["nonfinite"] = pg_norm2(self.theta, self.base[w], self.p[w], self.pg_current)
+            if poly and stale_threshold is not None and stale > stale_threshold:
+                info["dropped"] = True
+                infos.append(info)
+                continue
             wt = 1.0 if weights is None else weights[j]
+            if poly:
+                wt = poly_weight(stale)
             info["boundary"] = dn_arrive(self.theta, self.m, self.Delta, self.base[w], self.p[w], self.t, self.N,
                                          self.beta, self.eps, self.c, self.pg_current, wt, dc_lambda, buffered)
             self.t += 1

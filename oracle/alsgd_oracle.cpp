@@ -17,8 +17,9 @@
 //   orc_dylu        Eq. 6 values for speeds 1:1.5:2:3, H = 50.
 //   orc_lr_at       Eq. 3 end points and clamps.
 //   orc_schedule    Algorithm 2 + Algorithm 5 on hand timelines (Fig. 3 description).
-//   orc_poly_weight, delay compensation, buffered mode: formulas of Section 4 ("Existing Fixes");
-//                   parity unpinned beyond brute force on tiny inputs.
+//   orc_poly_weight, weight / dc_lambda / buffered arguments of orc_dn_arrive: formulas of Section 4
+//                   ("Existing Fixes"): hand cases, zero-drift and homogeneity properties, buffered
+//                   N = 1 == Eq. 4, buffered == Delayed Nesterov at cycle ends.
 #include <cmath>
 #include <cstdint>
 #include <cstring>
