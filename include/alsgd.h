@@ -72,6 +72,8 @@ typedef struct alsgd_ctx alsgd_ctx;
 
 #define ALSGD_CFG_REPLICA_BF16 1u  /* keep a bf16 copy of every worker's parameters */
 #define ALSGD_CFG_GRAD_STAGING 2u  /* reserve a P-element fp32 staging buffer so that alsgd_inner_adamw accepts host gradients */
+#define ALSGD_CFG_OUTER_BUFFERED 4u /* "Async. Buffer" of Section 4 instead of Delayed Nesterov: Delta accumulates every arrival,
+                                       theta and m move only on every N-th, by the Nesterov step of Eq. 4 on Delta/N; c is unused */
 
 typedef struct alsgd_config {
     uint32_t n_workers;  /* W >= 1 replicas resident in the arena */
@@ -141,7 +143,7 @@ typedef struct alsgd_arrival_info {
     uint32_t worker;
     uint32_t boundary;   /* 1 if (t+1) % N == 0: momentum updated, buffer reset */
     uint32_t nonfinite;  /* 1 if any entry was NaN or Inf (0 unless NANCHECK) */
-    uint32_t reserved;
+    uint32_t dropped;    /* 1 if the update was discarded as too stale (alsgd_arrive_ex, ALSGD_STALE_POLY_THRES) */
 } alsgd_arrival_info;
 
 /* The sync() of Algorithm 2 for the k workers of one grace window, in the given order: for each,
@@ -157,6 +159,28 @@ typedef struct alsgd_arrival_info {
  * worker that is not currently dispatched (never pulled, or already arrived and not re-dispatched). */
 int alsgd_arrive(alsgd_ctx* ctx, const uint32_t* worker_ids, uint32_t k, uint32_t flags,
                  alsgd_arrival_info* info);
+
+/* Staleness handling of Section 4 ("Existing Fixes"), staleness = server updates since the worker's dispatch. */
+#define ALSGD_STALE_NONE 0u
+#define ALSGD_STALE_POLY 1u        /* g <- (1 + staleness)^-0.5 * g  ("Async. DiLoCo + Poly") */
+#define ALSGD_STALE_POLY_THRES 2u  /* Poly, and updates with staleness > stale_threshold are discarded ("PolyThres") */
+
+typedef struct alsgd_arrive_opts {
+    const float* weights;      /* host, k entries or NULL: g_j <- weights[j] * g_j (ignored when a staleness rule is set) */
+    float dc_lambda;           /* delay compensation (Section 4): g <- g + lambda * g*g*(theta_now - theta_at_dispatch); 0 = off */
+    uint32_t staleness_rule;   /* ALSGD_STALE_* */
+    uint32_t stale_threshold;  /* for ALSGD_STALE_POLY_THRES (the paper uses 10) */
+    uint32_t reserved;
+} alsgd_arrive_opts;
+
+/* alsgd_arrive with the pseudo-gradient modifications of Section 4.  The pseudo-gradient of each arrival is
+ * first delay-compensated, then weighted, then enters Algorithm 3 (or the buffered outer step) unchanged
+ * otherwise; NORM / NANCHECK report the unmodified pseudo-gradient.  A discarded update (PolyThres) is not a
+ * server update: t does not advance, info[j].dropped = 1, and with RESEED its worker is still re-dispatched.
+ * opts == NULL behaves exactly like alsgd_arrive.  ALSGD_E_ARG: negative or non-finite dc_lambda, unknown
+ * staleness rule, non-finite weight. */
+int alsgd_arrive_ex(alsgd_ctx* ctx, const uint32_t* worker_ids, uint32_t k, uint32_t flags,
+                    const alsgd_arrive_opts* opts, alsgd_arrival_info* info);
 
 /* Server update counter t of Algorithm 3 and its phase t % N.  Either pointer may be NULL. */
 int alsgd_counters(alsgd_ctx* ctx, uint64_t* t_out, uint32_t* phase_out);

@@ -226,12 +226,13 @@ class OracleServer:
         for j, w in enumerate(ids):
             stale = self.t - self.pull_tick[w]
             info = {"worker": w, "tick": self.t, "staleness": stale, "dropped": False, "boundary": False}
-            if norm:
-                info["gnorm2"], info["nonfinite"] = pg_norm2(self.theta, self.base[w], self.p[w], self.pg_current)
             if poly and stale_threshold is not None and stale > stale_threshold:
-                info["dropped"] = True
+                info["dropped"] = True                 # never looked at: no diagnostics either
+                info["gnorm2"], info["nonfinite"] = 0.0, 0
                 infos.append(info)
                 continue
+            if norm:
+                info["gnorm2"], info["nonfinite"] = pg_norm2(self.theta, self.base[w], self.p[w], self.pg_current)
             wt = 1.0 if weights is None else weights[j]
             if poly:
                 wt = poly_weight(stale)

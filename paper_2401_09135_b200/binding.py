@@ -16,7 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libalsgd.so")
 OK, E_ARG, E_RANGE, E_STATE, E_CUDA, E_NOMEM, E_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
 TENSOR_DECAY = 1
 PG_DISPATCH, PG_CURRENT = 0, 1
-CFG_REPLICA_BF16, CFG_GRAD_STAGING = 1, 2
+CFG_REPLICA_BF16, CFG_GRAD_STAGING, CFG_OUTER_BUFFERED = 1, 2, 4
+STALE_NONE, STALE_POLY, STALE_POLY_THRES = 0, 1, 2
 ARRIVE_RESEED, ARRIVE_NORM, ARRIVE_NANCHECK = 1, 2, 4
 
 
@@ -33,7 +34,12 @@ class Config(C.Structure):
 
 class ArrivalInfo(C.Structure):
     _fields_ = [("tick", C.c_uint64), ("staleness", C.c_uint64), ("gnorm2", C.c_double),
-                ("worker", C.c_uint32), ("boundary", C.c_uint32), ("nonfinite", C.c_uint32), ("reserved", C.c_uint32)]
+                ("worker", C.c_uint32), ("boundary", C.c_uint32), ("nonfinite", C.c_uint32), ("dropped", C.c_uint32)]
+
+
+class ArriveOpts(C.Structure):
+    _fields_ = [("weights", C.POINTER(C.c_float)), ("dc_lambda", C.c_float), ("staleness_rule", C.c_uint32),
+                ("stale_threshold", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class Ptrs(C.Structure):
@@ -69,6 +75,7 @@ SIGNATURES = {
     "alsgd_pull": (C.c_int, [_vp, C.c_uint32]),
     "alsgd_inner_adamw": (C.c_int, [_vp, C.c_uint32, _vp, C.c_int, C.c_uint64, C.c_float]),
     "alsgd_arrive": (C.c_int, [_vp, _u32p, C.c_uint32, C.c_uint32, C.POINTER(ArrivalInfo)]),
+    "alsgd_arrive_ex": (C.c_int, [_vp, _u32p, C.c_uint32, C.c_uint32, C.POINTER(ArriveOpts), C.POINTER(ArrivalInfo)]),
     "alsgd_counters": (C.c_int, [_vp, _u64p, _u32p]),
     "alsgd_state_ptrs": (C.c_int, [_vp, C.POINTER(Ptrs)]),
     "alsgd_worker_state_ptrs": (C.c_int, [_vp, C.c_uint32, C.POINTER(WorkerPtrs)]),
@@ -196,7 +203,7 @@ class Context:
 
     def __init__(self, tensors, n_workers, N, beta, outer_lr, c=0.0, pg_base=PG_DISPATCH,
                  adam=(0.9, 0.95, 1e-8, 0.1), replica=True, grad_staging=False, align_elems=128,
-                 device=0, stream=None):
+                 device=0, stream=None, buffered=False):
         import torch
         self.torch = torch
         if not torch.cuda.is_available():
@@ -207,7 +214,8 @@ class Context:
         self.P, self.offsets = alsgd_layout_size(tensors, self.align)
         cfg = Config()
         cfg.n_workers, cfg.N, cfg.pg_base = int(n_workers), int(N), int(pg_base)
-        cfg.flags = (CFG_REPLICA_BF16 if replica else 0) | (CFG_GRAD_STAGING if grad_staging else 0)
+        cfg.flags = ((CFG_REPLICA_BF16 if replica else 0) | (CFG_GRAD_STAGING if grad_staging else 0)
+                     | (CFG_OUTER_BUFFERED if buffered else 0))
         cfg.beta, cfg.outer_lr, cfg.c = float(beta), float(outer_lr), float(c)
         cfg.adam_b1, cfg.adam_b2, cfg.adam_eps, cfg.adam_wd = [float(x) for x in adam]
         cfg.device = device
@@ -281,16 +289,30 @@ class Context:
         a, d = self._ptr(grads)
         _check(lib().alsgd_inner_adamw(self._h, int(w), a, d, int(step), float(lr)), "alsgd_inner_adamw", self._h)
 
+    @staticmethod
+    def _infos(info, k):
+        return [{"worker": int(i.worker), "tick": int(i.tick), "staleness": int(i.staleness),
+                 "boundary": bool(i.boundary), "gnorm2": float(i.gnorm2), "nonfinite": int(i.nonfinite),
+                 "dropped": bool(i.dropped)} for i in info[:k]]
+
     def alsgd_arrive(self, worker_ids, flags=ARRIVE_RESEED, want_info=True):
         k = len(worker_ids)
         ids = (C.c_uint32 * max(k, 1))(*[int(x) for x in worker_ids])
         info = (ArrivalInfo * max(k, 1))() if want_info else None
         _check(lib().alsgd_arrive(self._h, ids, k, int(flags), info), "alsgd_arrive", self._h)
-        if not want_info:
-            return None
-        return [{"worker": int(i.worker), "tick": int(i.tick), "staleness": int(i.staleness),
-                 "boundary": bool(i.boundary), "gnorm2": float(i.gnorm2), "nonfinite": int(i.nonfinite)}
-                for i in info[:k]]
+        return self._infos(info, k) if want_info else None
+
+    def alsgd_arrive_ex(self, worker_ids, flags=ARRIVE_RESEED, weights=None, dc_lambda=0.0,
+                        staleness_rule=STALE_NONE, stale_threshold=0, want_info=True):
+        k = len(worker_ids)
+        ids = (C.c_uint32 * max(k, 1))(*[int(x) for x in worker_ids])
+        info = (ArrivalInfo * max(k, 1))() if want_info else None
+        opts = ArriveOpts()
+        wbuf = (C.c_float * max(k, 1))(*[float(x) for x in weights]) if weights is not None else None
+        opts.weights = wbuf
+        opts.dc_lambda, opts.staleness_rule, opts.stale_threshold = float(dc_lambda), int(staleness_rule), int(stale_threshold)
+        _check(lib().alsgd_arrive_ex(self._h, ids, k, int(flags), C.byref(opts), info), "alsgd_arrive_ex", self._h)
+        return self._infos(info, k) if want_info else None
 
     def alsgd_counters(self):
         t, ph = C.c_uint64(), C.c_uint32()

@@ -76,7 +76,7 @@ bool valid_cfg(const alsgd_config* c) {
     if (!c) return false;
     if (c->n_workers == 0 || c->N == 0) return false;
     if (c->pg_base != ALSGD_PG_DISPATCH && c->pg_base != ALSGD_PG_CURRENT) return false;
-    if (c->flags & ~(ALSGD_CFG_REPLICA_BF16 | ALSGD_CFG_GRAD_STAGING)) return false;
+    if (c->flags & ~(ALSGD_CFG_REPLICA_BF16 | ALSGD_CFG_GRAD_STAGING | ALSGD_CFG_OUTER_BUFFERED)) return false;
     if (!(c->beta >= 0.0f && c->beta < 1.0f)) return false;
     if (!std::isfinite(c->outer_lr)) return false;
     if (!(c->c >= 0.0f && (double)c->c * (double)c->N <= 1.0 + 1e-6)) return false;
@@ -312,7 +312,7 @@ int alsgd_pull(alsgd_ctx* c, uint32_t worker) {
     a.n_seed = 1;
     fill_seed(a, 0, w);
     DeviceGuard g(c->cfg.device);
-    ALSGD_CUDA(c, launch_arrive(a, false, false, c->lc, c->stream));
+    ALSGD_CUDA(c, launch_arrive(a, false, false, false, c->lc, c->stream));
     w.pull_tick = c->t;
     w.state = kDispatched;
     return ALSGD_OK;
@@ -346,9 +346,25 @@ int alsgd_inner_adamw(alsgd_ctx* c, uint32_t worker, const float* grads, int gra
     return ALSGD_OK;
 }
 
-int alsgd_arrive(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, alsgd_arrival_info* info) {
+}  // extern "C"
+
+namespace {
+
+struct ArrivalPlan {
+    uint64_t tick = 0;       // Algorithm 3's t this arrival is applied at (or would have been)
+    uint64_t staleness = 0;
+    float weight = 1.0f;
+    bool dropped = false;
+};
+
+int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, const alsgd_arrive_opts* opts,
+                alsgd_arrival_info* info) {
     if (!c) return ALSGD_E_ARG;
     if (flags & ~(ALSGD_ARRIVE_RESEED | ALSGD_ARRIVE_NORM | ALSGD_ARRIVE_NANCHECK)) return ALSGD_E_ARG;
+    if (opts) {
+        if (!(opts->dc_lambda >= 0.0f) || !std::isfinite(opts->dc_lambda)) return ALSGD_E_ARG;
+        if (opts->staleness_rule > ALSGD_STALE_POLY_THRES) return ALSGD_E_ARG;
+    }
     if (k == 0) return ALSGD_OK;
     if (!ids) return ALSGD_E_ARG;
     const uint32_t W = c->cfg.n_workers;
@@ -365,38 +381,71 @@ int alsgd_arrive(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, 
     const bool diag = (flags & (ALSGD_ARRIVE_NORM | ALSGD_ARRIVE_NANCHECK)) != 0;
     const bool reseed = (flags & ALSGD_ARRIVE_RESEED) != 0;
     const bool current = c->cfg.pg_base == ALSGD_PG_CURRENT;
+    const bool buffered = (c->cfg.flags & ALSGD_CFG_OUTER_BUFFERED) != 0;
     const uint32_t N = c->cfg.N;
+    const uint32_t rule = opts ? opts->staleness_rule : ALSGD_STALE_NONE;
+    const float dc_lambda = opts ? opts->dc_lambda : 0.0f;
+
+    // ---- host plan: ticks, staleness, weights, discarded updates (Section 4, Poly / PolyThres)
+    std::vector<ArrivalPlan> plan(k);
+    std::vector<uint32_t> active;      // indices into ids[] of the arrivals that reach the kernel
+    uint64_t t = c->t;
+    bool extended = buffered || dc_lambda != 0.0f;
+    for (uint32_t j = 0; j < k; ++j) {
+        ArrivalPlan& a = plan[j];
+        a.tick = t;
+        a.staleness = t - c->workers[ids[j]].pull_tick;
+        if (rule == ALSGD_STALE_POLY_THRES && a.staleness > opts->stale_threshold) { a.dropped = true; continue; }
+        if (rule != ALSGD_STALE_NONE) a.weight = (float)std::pow(1.0 + (double)a.staleness, -0.5);
+        else if (opts && opts->weights) a.weight = opts->weights[j];
+        if (!std::isfinite(a.weight)) return ALSGD_E_ARG;
+        if (a.weight != 1.0f) extended = true;
+        active.push_back(j);
+        ++t;
+    }
+    const uint32_t ka = (uint32_t)active.size();
     DeviceGuard g(c->cfg.device);
 
     // Everything below only enqueues; the bookkeeping is committed after the last launch succeeded.
-    uint64_t t = c->t;
     bool delta_zero = c->delta_zero, delta_stored = c->delta_stored;
     std::vector<double> norms(k, 0.0);
     std::vector<unsigned int> bads(k, 0u);
 
-    const uint32_t n_chunks = (k + kMaxArrivals - 1) / kMaxArrivals;
+    const uint32_t n_chunks = (ka + kMaxArrivals - 1) / kMaxArrivals;
     uint32_t seeded = 0;  // how many of the last ids[] the final arrival launch re-seeds itself
     for (uint32_t ch = 0; ch < n_chunks; ++ch) {
         const uint32_t j0 = ch * kMaxArrivals;
-        const uint32_t kk = (k - j0 < (uint32_t)kMaxArrivals) ? k - j0 : (uint32_t)kMaxArrivals;
+        const uint32_t kk = (ka - j0 < (uint32_t)kMaxArrivals) ? ka - j0 : (uint32_t)kMaxArrivals;
         ArriveArgs a{};
         a.theta = c->theta; a.delta = c->delta; a.mom = c->mom;
         a.gnorm2 = c->gnorm2; a.nonfinite = c->nonfinite;
         a.n = c->P;
         a.n_arr = kk;
         a.beta = c->cfg.beta; a.eps = c->cfg.outer_lr; a.inv_n = c->inv_n; a.cb = c->cb; a.cn = c->cn;
+        a.dc_lambda = dc_lambda;
+        a.beta2 = c->cfg.beta * c->cfg.beta;
+        a.one_plus_beta = 1.0f + c->cfg.beta;
         bool any_boundary = false, last_boundary = false;
         for (uint32_t j = 0; j < kk; ++j) {
-            const Worker& w = c->workers[ids[j0 + j]];
+            const uint32_t src = active[j0 + j];
+            const Worker& w = c->workers[ids[src]];
             a.p[j] = w.p;
             a.base[j] = w.base;
-            const bool b = ((t + j + 1) % N) == 0;          // Algorithm 3's boundary test
+            a.w[j] = plan[src].weight;
+            const bool b = ((plan[src].tick + 1) % N) == 0;          // Algorithm 3's boundary test
             if (b) { a.boundary_mask |= 1u << j; any_boundary = true; }
             last_boundary = b;
         }
+        for (uint32_t j = kk; j < (uint32_t)kMaxArrivals; ++j) a.w[j] = 1.0f;
         if (delta_zero) a.flags |= kDeltaZeroIn;
         if (last_boundary) a.flags |= kDeltaSkipStore;
-        if (c->cfg.c != 0.0f) a.flags |= kCNonZero | kReadM;
+        if (buffered) {
+            a.flags |= kBuffered;
+            if (!any_boundary) a.flags |= kSkipThetaStore;
+        } else if (c->cfg.c != 0.0f) {
+            a.flags |= kCNonZero | kReadM;
+        }
+        if (dc_lambda != 0.0f) a.flags |= kDelayComp;
         if (any_boundary) a.flags |= kReadM | kWriteM;
         if (reseed && ch + 1 == n_chunks) {               // the final theta exists only in the last pass
             const uint32_t ns = k < (uint32_t)kMaxSeeds ? k : (uint32_t)kMaxSeeds;
@@ -408,17 +457,20 @@ int alsgd_arrive(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, 
             ALSGD_CUDA(c, cudaMemsetAsync(c->gnorm2, 0, sizeof(double) * kMaxArrivals, c->stream));
             ALSGD_CUDA(c, cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * kMaxArrivals, c->stream));
         }
-        ALSGD_CUDA(c, launch_arrive(a, current, diag, c->lc, c->stream));
+        ALSGD_CUDA(c, launch_arrive(a, current, diag, extended, c->lc, c->stream));
         if (diag && info) {
-            ALSGD_CUDA(c, cudaMemcpyAsync(norms.data() + j0, c->gnorm2, sizeof(double) * kk, cudaMemcpyDeviceToHost, c->stream));
-            ALSGD_CUDA(c, cudaMemcpyAsync(bads.data() + j0, c->nonfinite, sizeof(unsigned int) * kk, cudaMemcpyDeviceToHost, c->stream));
+            double nb[kMaxArrivals];
+            unsigned int fb[kMaxArrivals];
+            ALSGD_CUDA(c, cudaMemcpyAsync(nb, c->gnorm2, sizeof(double) * kk, cudaMemcpyDeviceToHost, c->stream));
+            ALSGD_CUDA(c, cudaMemcpyAsync(fb, c->nonfinite, sizeof(unsigned int) * kk, cudaMemcpyDeviceToHost, c->stream));
             ALSGD_CUDA(c, cudaStreamSynchronize(c->stream));
+            for (uint32_t j = 0; j < kk; ++j) { norms[active[j0 + j]] = nb[j]; bads[active[j0 + j]] = fb[j]; }
         }
-        t += kk;
         delta_zero = last_boundary;
         delta_stored = !last_boundary;
     }
-    // A batch larger than one launch can re-seed: the remaining workers get the same final theta.
+    // Workers the arrival launches did not re-seed (a batch larger than one launch, or nothing but
+    // discarded updates): the same final theta through standalone pulls.
     if (reseed && seeded < k) {
         uint32_t left = k - seeded, at = 0;
         while (left) {
@@ -426,7 +478,7 @@ int alsgd_arrive(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, 
             ArriveArgs a{};
             a.theta = c->theta; a.n = c->P; a.n_seed = ns;
             for (uint32_t s = 0; s < ns; ++s) fill_seed(a, s, c->workers[ids[at + s]]);
-            ALSGD_CUDA(c, launch_arrive(a, false, false, c->lc, c->stream));
+            ALSGD_CUDA(c, launch_arrive(a, false, false, false, c->lc, c->stream));
             at += ns; left -= ns;
         }
     }
@@ -435,13 +487,13 @@ int alsgd_arrive(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, 
     if (info) {
         for (uint32_t j = 0; j < k; ++j) {
             alsgd_arrival_info& o = info[j];
-            o.tick = c->t + j;
-            o.staleness = o.tick - c->workers[ids[j]].pull_tick;
+            o.tick = plan[j].tick;
+            o.staleness = plan[j].staleness;
             o.worker = ids[j];
-            o.boundary = ((c->t + j + 1) % N) == 0 ? 1u : 0u;
+            o.dropped = plan[j].dropped ? 1u : 0u;
+            o.boundary = (!plan[j].dropped && ((plan[j].tick + 1) % N) == 0) ? 1u : 0u;
             o.gnorm2 = (flags & ALSGD_ARRIVE_NORM) ? norms[j] : 0.0;
             o.nonfinite = (flags & ALSGD_ARRIVE_NANCHECK) ? (bads[j] ? 1u : 0u) : 0u;
-            o.reserved = 0;
         }
     }
     c->t = t;
@@ -453,6 +505,19 @@ int alsgd_arrive(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, 
         else w.state = kArrived;
     }
     return ALSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int alsgd_arrive(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, alsgd_arrival_info* info) {
+    return arrive_impl(c, ids, k, flags, nullptr, info);
+}
+
+int alsgd_arrive_ex(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, const alsgd_arrive_opts* opts,
+                    alsgd_arrival_info* info) {
+    return arrive_impl(c, ids, k, flags, opts, info);
 }
 
 int alsgd_counters(alsgd_ctx* c, uint64_t* t_out, uint32_t* phase_out) {

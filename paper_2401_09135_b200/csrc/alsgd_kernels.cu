@@ -41,18 +41,37 @@ __device__ __forceinline__ uint2 bf16_pack4(const float4& x) {
 }
 
 // K sequential arrivals of Algorithm 3 on one element.  th, d, mm carry theta, Delta, momentum.
-template <int K, bool DIAG, bool CUR>
+// EXT adds the Section 4 variants: delay compensation, staleness weight, buffered outer step.
+template <int K, bool DIAG, bool CUR, bool EXT>
 __device__ __forceinline__ void dn_element(float& th, float& d, float& mm, const float* b, const float* p,
                                            const ArriveArgs& a, double* acc, uint32_t& bad) {
 #pragma unroll
     for (int j = 0; j < K; ++j) {
         const float start = CUR ? th : b[j];
-        const float g = start - p[j];                 // pseudo-gradient
+        float g = start - p[j];                       // pseudo-gradient
         if (DIAG) {
             acc[j] += (double)g * (double)g;
             if (!isfinite(g)) bad |= 1u << j;
         }
+        if (EXT) {
+            if (a.flags & kDelayComp) {               // g + lambda * g*g*(theta_now - theta_at_dispatch)
+                const float drift = th - start;
+                g = g + ((a.dc_lambda * (g * g)) * drift);
+            }
+            if (a.w[j] != 1.0f) g = a.w[j] * g;
+        }
         d = d + g;                                    // Delta <- Delta + g
+        if (EXT && (a.flags & kBuffered)) {
+            if ((a.boundary_mask >> j) & 1u) {        // Eq. 4 on the buffer mean
+                const float mean = d * a.inv_n;
+                const float mn = (a.beta * mm) + mean;
+                const float u = (a.beta2 * mm) + (a.one_plus_beta * mean);
+                th = th - (a.eps * u);
+                mm = mn;
+                d = 0.0f;
+            }
+            continue;
+        }
         const float gn = g * a.inv_n;                 // g / N
         if ((a.boundary_mask >> j) & 1u) {
             const float mn = (a.beta * mm) + (d * a.inv_n);   // m <- beta m + Delta/N
@@ -67,7 +86,7 @@ __device__ __forceinline__ void dn_element(float& th, float& d, float& mm, const
     }
 }
 
-template <int K, int V, bool DIAG, bool CUR>
+template <int K, int V, bool DIAG, bool CUR, bool EXT>
 __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ ArriveArgs a) {
     constexpr int KK = K > 0 ? K : 1;
     const uint64_t nvec = a.n >> 2;
@@ -77,6 +96,7 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
     const bool write_delta = K > 0 && !(flags & kDeltaSkipStore);
     const bool read_m = K > 0 && (flags & kReadM);
     const bool write_m = K > 0 && (flags & kWriteM);
+    const bool write_theta = !(EXT && (flags & kSkipThetaStore));
     const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
 
     double acc[KK];
@@ -123,9 +143,9 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
                         pe[j] = reinterpret_cast<const float*>(&p[j][v])[e];
                         be[j] = CUR ? 0.f : reinterpret_cast<const float*>(&b[j][v])[e];
                     }
-                    dn_element<K, DIAG, CUR>(thf[e], df[e], mf[e], be, pe, a, acc, bad);
+                    dn_element<K, DIAG, CUR, EXT>(thf[e], df[e], mf[e], be, pe, a, acc, bad);
                 }
-                st_stream(theta4 + i, th[v]);
+                if (write_theta) st_stream(theta4 + i, th[v]);
                 if (write_delta) st_stream(delta4 + i, d[v]);
                 if (write_m) st_stream(mom4 + i, mm[v]);
             }
@@ -157,8 +177,8 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
                 pe[j] = a.p[j][i];
                 be[j] = CUR ? 0.f : a.base[j][i];
             }
-            dn_element<K, DIAG, CUR>(th, d, mm, be, pe, a, acc, bad);
-            a.theta[i] = th;
+            dn_element<K, DIAG, CUR, EXT>(th, d, mm, be, pe, a, acc, bad);
+            if (write_theta) a.theta[i] = th;
             if (write_delta) a.delta[i] = d;
             if (write_m) a.mom[i] = mm;
         }
@@ -321,10 +341,10 @@ cudaError_t grid_for(uint64_t n, int vecs_per_thread, unsigned* grid) {
 // K=1: V=1 6635, V=2 6693, V=4 6735;  K=2: V=1 6612, V=2 6689;  K=4: V=1 6576, V=2 6626;  K=8: V=1 6600.
 constexpr int arrive_vecs(int K) { return K <= 1 ? 4 : (K <= 4 ? 2 : 1); }
 
-template <int K, bool DIAG, bool CUR>
+template <int K, bool DIAG, bool CUR, bool EXT>
 cudaError_t launch_arrive_k(const ArriveArgs& a, const LaunchCfg& lc, cudaStream_t s) {
     constexpr int V = arrive_vecs(K);
-    auto kern = arrive_kernel<K, V, DIAG, CUR>;
+    auto kern = arrive_kernel<K, V, DIAG, CUR, EXT>;
     unsigned grid = 1;
     cudaError_t e = grid_for(a.n, V, &grid);
     if (e != cudaSuccess) return e;
@@ -333,29 +353,34 @@ cudaError_t launch_arrive_k(const ArriveArgs& a, const LaunchCfg& lc, cudaStream
     return cudaGetLastError();
 }
 
-template <bool DIAG, bool CUR>
+template <bool DIAG, bool CUR, bool EXT>
 cudaError_t launch_arrive_dc(const ArriveArgs& a, const LaunchCfg& lc, cudaStream_t s) {
     switch (a.n_arr) {
-        case 0: return launch_arrive_k<0, false, false>(a, lc, s);
-        case 1: return launch_arrive_k<1, DIAG, CUR>(a, lc, s);
-        case 2: return launch_arrive_k<2, DIAG, CUR>(a, lc, s);
-        case 3: return launch_arrive_k<3, DIAG, CUR>(a, lc, s);
-        case 4: return launch_arrive_k<4, DIAG, CUR>(a, lc, s);
-        case 5: return launch_arrive_k<5, DIAG, CUR>(a, lc, s);
-        case 6: return launch_arrive_k<6, DIAG, CUR>(a, lc, s);
-        case 7: return launch_arrive_k<7, DIAG, CUR>(a, lc, s);
-        case 8: return launch_arrive_k<8, DIAG, CUR>(a, lc, s);
+        case 0: return launch_arrive_k<0, false, false, false>(a, lc, s);
+        case 1: return launch_arrive_k<1, DIAG, CUR, EXT>(a, lc, s);
+        case 2: return launch_arrive_k<2, DIAG, CUR, EXT>(a, lc, s);
+        case 3: return launch_arrive_k<3, DIAG, CUR, EXT>(a, lc, s);
+        case 4: return launch_arrive_k<4, DIAG, CUR, EXT>(a, lc, s);
+        case 5: return launch_arrive_k<5, DIAG, CUR, EXT>(a, lc, s);
+        case 6: return launch_arrive_k<6, DIAG, CUR, EXT>(a, lc, s);
+        case 7: return launch_arrive_k<7, DIAG, CUR, EXT>(a, lc, s);
+        case 8: return launch_arrive_k<8, DIAG, CUR, EXT>(a, lc, s);
         default: return cudaErrorInvalidValue;
     }
 }
 
+template <bool DIAG, bool CUR>
+cudaError_t launch_arrive_e(const ArriveArgs& a, bool extended, const LaunchCfg& lc, cudaStream_t s) {
+    return extended ? launch_arrive_dc<DIAG, CUR, true>(a, lc, s) : launch_arrive_dc<DIAG, CUR, false>(a, lc, s);
+}
+
 }  // namespace
 
-cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, const LaunchCfg& lc, cudaStream_t s) {
+cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, bool extended, const LaunchCfg& lc, cudaStream_t s) {
     if (a.n == 0) return cudaSuccess;
     if (a.n_arr > (uint32_t)kMaxArrivals || a.n_seed > (uint32_t)kMaxSeeds) return cudaErrorInvalidValue;
-    if (diagnostics) return pg_current ? launch_arrive_dc<true, true>(a, lc, s) : launch_arrive_dc<true, false>(a, lc, s);
-    return pg_current ? launch_arrive_dc<false, true>(a, lc, s) : launch_arrive_dc<false, false>(a, lc, s);
+    if (diagnostics) return pg_current ? launch_arrive_e<true, true>(a, extended, lc, s) : launch_arrive_e<true, false>(a, extended, lc, s);
+    return pg_current ? launch_arrive_e<false, true>(a, extended, lc, s) : launch_arrive_e<false, false>(a, extended, lc, s);
 }
 
 cudaError_t launch_adamw(const AdamArgs& a, const LaunchCfg& lc, cudaStream_t s) {

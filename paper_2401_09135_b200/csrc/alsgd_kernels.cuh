@@ -13,7 +13,10 @@ enum : uint32_t {
     kDeltaSkipStore = 2u,  // Delta is zero by definition on exit: do not write it
     kReadM = 4u,           // momentum is needed (a boundary in the batch, or c != 0)
     kWriteM = 8u,          // momentum changes (a boundary in the batch)
-    kCNonZero = 16u        // momentum activation c != 0
+    kCNonZero = 16u,       // momentum activation c != 0
+    kDelayComp = 32u,      // delay compensation on the pseudo-gradient (dc_lambda != 0)
+    kBuffered = 64u,       // buffered outer step: theta and m move only at a boundary, by Eq. 4 on Delta/N
+    kSkipThetaStore = 128u // theta is unchanged by this launch (buffered, no boundary): do not write it
 };
 
 // One batch of arrivals of Algorithm 3 plus the re-seed of the workers that are dispatched again.
@@ -34,6 +37,10 @@ struct ArriveArgs {
     uint32_t boundary_mask;           // bit j: arrival j is a momentum boundary
     uint32_t flags;
     float beta, eps, inv_n, cb, cn;
+    // extended path only (weights, delay compensation, buffered outer step)
+    float w[kMaxArrivals];            // staleness weights (1 = none)
+    float dc_lambda;
+    float beta2, one_plus_beta;       // beta*beta and 1+beta, each one fp32 operation
 };
 
 struct AdamArgs {
@@ -53,7 +60,7 @@ struct LaunchCfg {
     int sm_count;
 };
 
-cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, const LaunchCfg& lc, cudaStream_t s);
+cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, bool extended, const LaunchCfg& lc, cudaStream_t s);
 cudaError_t launch_adamw(const AdamArgs& a, const LaunchCfg& lc, cudaStream_t s);
 
 }  // namespace alsgd

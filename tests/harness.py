@@ -45,13 +45,15 @@ def assert_fp32(name, got, ref, strict=True):
 
 class Pair:
     def __init__(self, tensors, n_workers, N, beta, outer_lr, c=0.0, pg_current=False, replica=True,
-                 adam=(0.9, 0.95, 1e-8, 0.1), align=128, n_sample=None, grad_staging=False, strict=True):
+                 adam=(0.9, 0.95, 1e-8, 0.1), align=128, n_sample=None, grad_staging=False, strict=True,
+                 buffered=False):
         self.tensors = tensors
         self.W = n_workers
         self.strict = strict
         self.ctx = B.Context(tensors, n_workers, N, beta, outer_lr, c=c,
                              pg_base=B.PG_CURRENT if pg_current else B.PG_DISPATCH, adam=adam, replica=replica,
-                             grad_staging=grad_staging, align_elems=align)
+                             grad_staging=grad_staging, align_elems=align, buffered=buffered)
+        self.buffered = buffered
         self.P, self.offsets = self.ctx.P, self.ctx.offsets
         o_offs, o_P = oracle.layout_offsets([t.numel for t in tensors], align)
         assert (o_P, o_offs) == (self.P, self.offsets)
@@ -101,13 +103,23 @@ class Pair:
         self.ctx.alsgd_inner_adamw(w, g_dev, step, lr)
         self.orc.inner_adamw(w, self.take(g_np), step, lr)
 
-    def arrive(self, ids, reseed=True, norm=False):
+    def arrive(self, ids, reseed=True, norm=False, weights=None, dc_lambda=0.0, poly=False, stale_threshold=None):
         flags = (B.ARRIVE_RESEED if reseed else 0) | ((B.ARRIVE_NORM | B.ARRIVE_NANCHECK) if norm else 0)
-        got = self.ctx.alsgd_arrive(ids, flags)
-        ref = self.orc.arrive(ids, reseed_after=reseed, norm=norm and self.idx is None)
+        plain = weights is None and dc_lambda == 0.0 and not poly
+        if plain:
+            got = self.ctx.alsgd_arrive(ids, flags)
+        else:
+            rule = B.STALE_NONE if not poly else (B.STALE_POLY if stale_threshold is None else B.STALE_POLY_THRES)
+            got = self.ctx.alsgd_arrive_ex(ids, flags, weights=weights, dc_lambda=dc_lambda, staleness_rule=rule,
+                                           stale_threshold=stale_threshold or 0)
+        w32 = None if weights is None else [float(np.float32(x)) for x in weights]
+        ref = self.orc.arrive(ids, reseed_after=reseed, norm=norm and self.idx is None, weights=w32,
+                              dc_lambda=float(np.float32(dc_lambda)), buffered=self.buffered, poly=poly,
+                              stale_threshold=stale_threshold)
         for g, r in zip(got, ref):                 # bookkeeping: bit-exact
             assert g["worker"] == r["worker"] and g["tick"] == r["tick"]
             assert g["boundary"] == r["boundary"] and g["staleness"] == r["staleness"]
+            assert g["dropped"] == r["dropped"]
             if norm and self.idx is None:
                 assert g["nonfinite"] == r["nonfinite"]
                 if not r["nonfinite"]:
