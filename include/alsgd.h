@@ -209,6 +209,19 @@ typedef struct alsgd_worker_ptrs {
 int alsgd_state_ptrs(alsgd_ctx* ctx, alsgd_ptrs* out);
 int alsgd_worker_state_ptrs(alsgd_ctx* ctx, uint32_t worker, alsgd_worker_ptrs* out);
 
+/* Checkpoint / resume.  The paper starts its runs from a pretrained checkpoint (Section 4; Table 5) and
+ * keeps each worker's optimizer state across rounds, without describing a mechanism; this is the
+ * library's.  The image holds the layout size, W, N, the pseudo-gradient mode, t, every worker's dispatch
+ * state and pull tick, then theta, m, Delta and each worker's parameters, snapshot, AdamW moments and replica.
+ *   alsgd_state_bytes     size of the image for this context
+ *   alsgd_export_state    host_dst: host, `bytes` >= that size; waits for the stream
+ *   alsgd_import_state    host_src: host image written by a context with the same layout size, W, N, mode
+ *                         and replica setting (hyper-parameters may differ); replaces the whole state; waits
+ * ALSGD_E_NOMEM: buffer too small.  ALSGD_E_ARG: not an image, or made for a different shape. */
+int alsgd_state_bytes(alsgd_ctx* ctx, uint64_t* bytes_out);
+int alsgd_export_state(alsgd_ctx* ctx, void* host_dst, uint64_t bytes);
+int alsgd_import_state(alsgd_ctx* ctx, const void* host_src, uint64_t bytes);
+
 /* Wait for the context's stream. */
 int alsgd_sync(alsgd_ctx* ctx);
 

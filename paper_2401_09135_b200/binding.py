@@ -79,6 +79,9 @@ SIGNATURES = {
     "alsgd_counters": (C.c_int, [_vp, _u64p, _u32p]),
     "alsgd_state_ptrs": (C.c_int, [_vp, C.POINTER(Ptrs)]),
     "alsgd_worker_state_ptrs": (C.c_int, [_vp, C.c_uint32, C.POINTER(WorkerPtrs)]),
+    "alsgd_state_bytes": (C.c_int, [_vp, _u64p]),
+    "alsgd_export_state": (C.c_int, [_vp, _vp, C.c_uint64]),
+    "alsgd_import_state": (C.c_int, [_vp, _vp, C.c_uint64]),
     "alsgd_sync": (C.c_int, [_vp]),
     "alsgd_last_cuda_error": (C.c_int, [_vp]),
     "alsgd_dylu_steps": (C.c_int, [_f64p, C.c_uint32, C.c_uint32, _u32p]),
@@ -318,6 +321,22 @@ class Context:
         t, ph = C.c_uint64(), C.c_uint32()
         _check(lib().alsgd_counters(self._h, C.byref(t), C.byref(ph)), "alsgd_counters", self._h)
         return int(t.value), int(ph.value)
+
+    def alsgd_state_bytes(self):
+        n = C.c_uint64()
+        _check(lib().alsgd_state_bytes(self._h, C.byref(n)), "alsgd_state_bytes", self._h)
+        return int(n.value)
+
+    def alsgd_export_state(self):
+        """The state image as a numpy uint8 array."""
+        import numpy as np
+        buf = np.empty(self.alsgd_state_bytes(), dtype=np.uint8)
+        _check(lib().alsgd_export_state(self._h, buf.ctypes.data, buf.size), "alsgd_export_state", self._h)
+        return buf
+
+    def alsgd_import_state(self, image):
+        assert image.dtype.name == "uint8" and image.flags["C_CONTIGUOUS"]
+        _check(lib().alsgd_import_state(self._h, image.ctypes.data, image.size), "alsgd_import_state", self._h)
 
     def alsgd_sync(self):
         _check(lib().alsgd_sync(self._h), "alsgd_sync", self._h)

@@ -547,6 +547,125 @@ int alsgd_worker_state_ptrs(alsgd_ctx* c, uint32_t worker, alsgd_worker_ptrs* ou
     return ALSGD_OK;
 }
 
+}  // extern "C"
+
+namespace {
+
+struct ImageHeader {
+    char magic[8];
+    uint32_t version;
+    uint32_t n_workers;
+    uint64_t P;
+    uint32_t N;
+    uint32_t pg_base;
+    uint32_t has_replica;
+    uint32_t delta_zero;
+    uint64_t t;
+};
+struct ImageWorker {
+    uint64_t pull_tick;
+    uint32_t state;
+    uint32_t reserved;
+};
+const char kMagic[8] = {'A', 'L', 'S', 'G', 'D', 'C', 'K', '1'};
+
+uint64_t image_bytes(const alsgd_ctx* c) {
+    const uint64_t P = c->P;
+    uint64_t per_worker = 3 * 4 * P;                               // p, adam m, adam v
+    if (c->workers[0].base) per_worker += 4 * P;
+    if (c->workers[0].rep) per_worker += 2 * P;
+    return sizeof(ImageHeader) + sizeof(ImageWorker) * c->cfg.n_workers + 3 * 4 * P + per_worker * c->cfg.n_workers;
+}
+
+// Visit every device slice in image order.
+template <typename F>
+int for_each_slice(alsgd_ctx* c, F f) {
+    const uint64_t P = c->P;
+    int rc;
+    if ((rc = f(c->theta, 4 * P)) || (rc = f(c->mom, 4 * P)) || (rc = f(c->delta, 4 * P))) return rc;
+    for (Worker& w : c->workers) {
+        if ((rc = f(w.p, 4 * P))) return rc;
+        if (w.base && (rc = f(w.base, 4 * P))) return rc;
+        if ((rc = f(w.am, 4 * P)) || (rc = f(w.av, 4 * P))) return rc;
+        if (w.rep && (rc = f(w.rep, 2 * P))) return rc;
+    }
+    return ALSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int alsgd_state_bytes(alsgd_ctx* c, uint64_t* bytes_out) {
+    if (!c || !bytes_out) return ALSGD_E_ARG;
+    *bytes_out = image_bytes(c);
+    return ALSGD_OK;
+}
+
+int alsgd_export_state(alsgd_ctx* c, void* host_dst, uint64_t bytes) {
+    if (!c || !host_dst) return ALSGD_E_ARG;
+    if (bytes < image_bytes(c)) return ALSGD_E_NOMEM;
+    DeviceGuard g(c->cfg.device);
+    if (c->delta_zero && !c->delta_stored) {                       // write out the zeros Delta stands for
+        ALSGD_CUDA(c, cudaMemsetAsync(c->delta, 0, sizeof(float) * c->P, c->stream));
+        c->delta_stored = true;
+    }
+    uint8_t* out = static_cast<uint8_t*>(host_dst);
+    ImageHeader h{};
+    std::memcpy(h.magic, kMagic, 8);
+    h.version = 1; h.n_workers = c->cfg.n_workers; h.P = c->P; h.N = c->cfg.N; h.pg_base = c->cfg.pg_base;
+    h.has_replica = c->workers[0].rep ? 1u : 0u; h.delta_zero = c->delta_zero ? 1u : 0u; h.t = c->t;
+    std::memcpy(out, &h, sizeof(h));
+    out += sizeof(h);
+    for (const Worker& w : c->workers) {
+        ImageWorker iw{w.pull_tick, (uint32_t)w.state, 0u};
+        std::memcpy(out, &iw, sizeof(iw));
+        out += sizeof(iw);
+    }
+    int rc = for_each_slice(c, [&](void* dev, uint64_t n) -> int {
+        if (cudaMemcpyAsync(out, dev, n, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess) return cuda_fail(c, cudaGetLastError());
+        out += n;
+        return ALSGD_OK;
+    });
+    if (rc != ALSGD_OK) return rc;
+    ALSGD_CUDA(c, cudaStreamSynchronize(c->stream));
+    return ALSGD_OK;
+}
+
+int alsgd_import_state(alsgd_ctx* c, const void* host_src, uint64_t bytes) {
+    if (!c || !host_src) return ALSGD_E_ARG;
+    if (bytes < sizeof(ImageHeader)) return ALSGD_E_ARG;
+    const uint8_t* in = static_cast<const uint8_t*>(host_src);
+    ImageHeader h;
+    std::memcpy(&h, in, sizeof(h));
+    if (std::memcmp(h.magic, kMagic, 8) != 0 || h.version != 1) return ALSGD_E_ARG;
+    if (h.P != c->P || h.n_workers != c->cfg.n_workers || h.N != c->cfg.N || h.pg_base != c->cfg.pg_base ||
+        h.has_replica != (c->workers[0].rep ? 1u : 0u)) return ALSGD_E_ARG;
+    if (bytes < image_bytes(c)) return ALSGD_E_ARG;
+    in += sizeof(h);
+    std::vector<ImageWorker> iw(c->cfg.n_workers);
+    std::memcpy(iw.data(), in, sizeof(ImageWorker) * iw.size());
+    for (const ImageWorker& w : iw)
+        if (w.state > (uint32_t)kArrived) return ALSGD_E_ARG;
+    in += sizeof(ImageWorker) * iw.size();
+    DeviceGuard g(c->cfg.device);
+    int rc = for_each_slice(c, [&](void* dev, uint64_t n) -> int {
+        if (cudaMemcpyAsync(dev, in, n, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return cuda_fail(c, cudaGetLastError());
+        in += n;
+        return ALSGD_OK;
+    });
+    if (rc != ALSGD_OK) return rc;
+    ALSGD_CUDA(c, cudaStreamSynchronize(c->stream));
+    c->t = h.t;
+    c->delta_zero = h.delta_zero != 0;
+    c->delta_stored = true;
+    for (uint32_t w = 0; w < c->cfg.n_workers; ++w) {
+        c->workers[w].pull_tick = iw[w].pull_tick;
+        c->workers[w].state = (WorkerState)iw[w].state;
+    }
+    return ALSGD_OK;
+}
+
 int alsgd_sync(alsgd_ctx* c) {
     if (!c) return ALSGD_E_ARG;
     DeviceGuard g(c->cfg.device);
