@@ -375,10 +375,11 @@ def main_ksweep(args):
         ev = ev[1:]                                        # first round is warm-up
         arr_ms = sum(a.elapsed_time(b) for a, b, _ in ev) / len(ev)
         adam_ms = sum(b.elapsed_time(c) for _, b, c in ev) / len(ev)
-        # one full cycle per round (N = W = 8): Delta read on all batches but the first, written on all but
-        # the last, m read+written once; per arrival 8 B of (base, p) reads and 10 B of re-seed writes
+        # one full cycle per round (N = W = 8): theta read+written per batch, Delta read on all batches but the
+        # first and written on all but the last, m read+written once; per batch k worker vectors and the one
+        # snapshot its workers share are read, k x (params 4 + bf16 2) and one new snapshot are written
         nb = W // k
-        arr_bytes = (4 * nb + 4 * (nb - 1) + 4 * nb + 4 * (nb - 1) + 8 + 18 * W) * P
+        arr_bytes = (8 * nb + 8 * (nb - 1) + 8 + nb * (4 * k + 4) + nb * (6 * k + 4)) * P
         adam_bytes = ADAMW_BYTES * P * W * inner
         out.append({"k": k, "arrival_ms_per_round": arr_ms, "arrival_gbs": arr_bytes / arr_ms / 1e6,
                     "arrival_frac": arr_bytes / arr_ms / 1e6 / peak, "arrival_bytes_per_param_per_arrival": arr_bytes / P / W,

@@ -196,7 +196,8 @@ typedef struct alsgd_ptrs {
 
 typedef struct alsgd_worker_ptrs {
     float* p;          /* device, P: the worker's parameters */
-    float* base;       /* device, P: dispatch snapshot (NULL in ALSGD_PG_CURRENT mode) */
+    float* base;       /* device, P: dispatch snapshot, read-only for the caller: workers dispatched in the same
+                          window share one (NULL in ALSGD_PG_CURRENT mode) */
     float* adam_m;     /* device, P */
     float* adam_v;     /* device, P */
     uint16_t* replica; /* device, P bf16 bit patterns (NULL without ALSGD_CFG_REPLICA_BF16) */

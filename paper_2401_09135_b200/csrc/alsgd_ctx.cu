@@ -19,7 +19,8 @@ enum WorkerState : uint8_t { kNever = 0, kDispatched = 1, kArrived = 2 };
 
 struct Worker {
     float* p = nullptr;
-    float* base = nullptr;
+    float* base = nullptr;       // the snapshot slot this worker was dispatched with (may be shared)
+    int slot = -1;
     float* am = nullptr;
     float* av = nullptr;
     uint16_t* rep = nullptr;
@@ -103,6 +104,10 @@ struct alsgd_ctx {
     float* delta = nullptr;
     float* grad_stage = nullptr;
     std::vector<Worker> workers;
+    // Dispatch snapshots: W slots of P floats.  Workers dispatched together (one grace window, one
+    // theta) share one slot, so the snapshot is written once per window and read once per batch.
+    std::vector<float*> slot_ptr;
+    std::vector<uint32_t> slot_ref;
     // Algorithm 3 bookkeeping
     uint64_t t = 0;
     bool delta_zero = true;     // Delta is zero by definition (start, or right after a boundary)
@@ -128,6 +133,8 @@ uint64_t carve(alsgd_ctx* c, void* arena, uint64_t P, const alsgd_config& cfg, u
         c->seg_end = seg_end; c->seg_decay = seg_decay; c->gnorm2 = gn; c->nonfinite = nf;
         c->theta = theta; c->mom = mom; c->delta = delta;
         c->workers.assign(cfg.n_workers, Worker());
+        c->slot_ptr.clear();
+        c->slot_ref.clear();
     }
     for (uint32_t w = 0; w < cfg.n_workers; ++w) {
         float* p = k.take<float>(P);
@@ -138,6 +145,7 @@ uint64_t carve(alsgd_ctx* c, void* arena, uint64_t P, const alsgd_config& cfg, u
         if (c) {
             Worker& W = c->workers[w];
             W.p = p; W.base = base; W.am = am; W.av = av; W.rep = rep;
+            if (base) { W.slot = (int)w; c->slot_ptr.push_back(base); c->slot_ref.push_back(1u); }
         }
     }
     float* stage = (cfg.flags & ALSGD_CFG_GRAD_STAGING) ? k.take<float>(P) : nullptr;
@@ -176,10 +184,38 @@ int copy_vec(alsgd_ctx* c, void* dst, const void* src, uint64_t bytes, bool host
     return ALSGD_OK;
 }
 
-void fill_seed(ArriveArgs& a, uint32_t slot, const Worker& w) {
+// Re-seed target: the worker's parameters and replica, plus (for one worker of the window) the
+// snapshot slot the whole window will share.
+void fill_seed(ArriveArgs& a, uint32_t slot, const Worker& w, float* snapshot) {
     a.seed_p[slot] = w.p;
-    a.seed_base[slot] = w.base;
+    a.seed_base[slot] = snapshot;
     a.seed_rep[slot] = w.rep;
+}
+
+// The slot that is free once the given workers have let go of theirs (-1 when the pseudo-gradient
+// is taken against the running theta and no snapshots exist).  At most W - k other workers hold a
+// slot, so one of the W slots is always free.
+int pick_slot(const alsgd_ctx* c, const uint32_t* ids, uint32_t k) {
+    if (c->slot_ptr.empty()) return -1;
+    std::vector<uint32_t> ref(c->slot_ref);
+    for (uint32_t j = 0; j < k; ++j) {
+        const int s = c->workers[ids[j]].slot;
+        if (s >= 0) --ref[s];
+    }
+    for (size_t s = 0; s < ref.size(); ++s)
+        if (ref[s] == 0) return (int)s;
+    return -1;
+}
+
+void commit_slot(alsgd_ctx* c, const uint32_t* ids, uint32_t k, int s) {
+    if (s < 0) return;
+    for (uint32_t j = 0; j < k; ++j) {
+        Worker& w = c->workers[ids[j]];
+        if (w.slot >= 0) --c->slot_ref[w.slot];
+        w.slot = s;
+        w.base = c->slot_ptr[s];
+        ++c->slot_ref[s];
+    }
 }
 
 }  // namespace
@@ -310,9 +346,11 @@ int alsgd_pull(alsgd_ctx* c, uint32_t worker) {
     a.n = c->P;
     a.n_arr = 0;
     a.n_seed = 1;
-    fill_seed(a, 0, w);
+    const int slot = pick_slot(c, &worker, 1);
+    fill_seed(a, 0, w, slot >= 0 ? c->slot_ptr[slot] : nullptr);
     DeviceGuard g(c->cfg.device);
     ALSGD_CUDA(c, launch_arrive(a, false, false, false, c->lc, c->stream));
+    commit_slot(c, &worker, 1, slot);
     w.pull_tick = c->t;
     w.state = kDispatched;
     return ALSGD_OK;
@@ -413,6 +451,9 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
 
     const uint32_t n_chunks = (ka + kMaxArrivals - 1) / kMaxArrivals;
     uint32_t seeded = 0;  // how many of the last ids[] the final arrival launch re-seeds itself
+    const int new_slot = reseed ? pick_slot(c, ids, k) : -1;   // one snapshot for the whole window
+    float* snapshot = new_slot >= 0 ? c->slot_ptr[new_slot] : nullptr;
+    bool snapshot_written = false;
     for (uint32_t ch = 0; ch < n_chunks; ++ch) {
         const uint32_t j0 = ch * kMaxArrivals;
         const uint32_t kk = (ka - j0 < (uint32_t)kMaxArrivals) ? ka - j0 : (uint32_t)kMaxArrivals;
@@ -449,9 +490,10 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
         if (any_boundary) a.flags |= kReadM | kWriteM;
         if (reseed && ch + 1 == n_chunks) {               // the final theta exists only in the last pass
             const uint32_t ns = k < (uint32_t)kMaxSeeds ? k : (uint32_t)kMaxSeeds;
-            for (uint32_t s = 0; s < ns; ++s) fill_seed(a, s, c->workers[ids[k - ns + s]]);
+            for (uint32_t s = 0; s < ns; ++s) fill_seed(a, s, c->workers[ids[k - ns + s]], s == 0 ? snapshot : nullptr);
             a.n_seed = ns;
             seeded = ns;
+            snapshot_written = true;
         }
         if (diag) {
             ALSGD_CUDA(c, cudaMemsetAsync(c->gnorm2, 0, sizeof(double) * kMaxArrivals, c->stream));
@@ -477,7 +519,10 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
             const uint32_t ns = left < (uint32_t)kMaxSeeds ? left : (uint32_t)kMaxSeeds;
             ArriveArgs a{};
             a.theta = c->theta; a.n = c->P; a.n_seed = ns;
-            for (uint32_t s = 0; s < ns; ++s) fill_seed(a, s, c->workers[ids[at + s]]);
+            for (uint32_t s = 0; s < ns; ++s) {
+                fill_seed(a, s, c->workers[ids[at + s]], snapshot_written ? nullptr : snapshot);
+                snapshot_written = true;
+            }
             ALSGD_CUDA(c, launch_arrive(a, false, false, false, c->lc, c->stream));
             at += ns; left -= ns;
         }
@@ -499,6 +544,7 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
     c->t = t;
     c->delta_zero = delta_zero;
     c->delta_stored = delta_stored;
+    if (reseed) commit_slot(c, ids, k, new_slot);
     for (uint32_t j = 0; j < k; ++j) {
         Worker& w = c->workers[ids[j]];
         if (reseed) { w.state = kDispatched; w.pull_tick = c->t; }
@@ -649,6 +695,11 @@ int alsgd_import_state(alsgd_ctx* c, const void* host_src, uint64_t bytes) {
         if (w.state > (uint32_t)kArrived) return ALSGD_E_ARG;
     in += sizeof(ImageWorker) * iw.size();
     DeviceGuard g(c->cfg.device);
+    for (uint32_t w = 0; w < c->cfg.n_workers && !c->slot_ptr.empty(); ++w) {   // the image holds one snapshot per worker
+        c->workers[w].slot = (int)w;
+        c->workers[w].base = c->slot_ptr[w];
+        c->slot_ref[w] = 1u;
+    }
     int rc = for_each_slice(c, [&](void* dev, uint64_t n) -> int {
         if (cudaMemcpyAsync(dev, in, n, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return cuda_fail(c, cudaGetLastError());
         in += n;
