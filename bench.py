@@ -29,10 +29,10 @@ WORKLOAD = "decoder-110M(12L,d768,ff3072,V32000) W=4 N=4 beta=0.9 outer_lr=0.7 c
 SPEEDS = [1.0, 1.5, 2.0, 3.0]
 H = 50
 ADAMW_BYTES = 30          # g,p,m,v read (16) + p,m,v write (12) + bf16 replica write (2)
-ARRIVE_RESEED_BYTES = {   # theta, Delta, base, p read / theta, Delta write (+m on a boundary), + p, base, bf16 re-seed
-    "first": 20 + 10,     # Delta known zero: not read
-    "middle": 24 + 10,
-    "boundary": 28 + 10,  # + m read and write; Delta zero store elided
+ARRIVE_RESEED_BYTES = {   # theta, Delta, snapshot, p read / theta, Delta write (+m on a boundary), + new snapshot 4 and bf16 2
+    "first": 20 + 6,      # Delta known zero: not read
+    "middle": 24 + 6,     # (the re-seeded parameters are not stored twice: until the worker's next AdamW step
+    "boundary": 28 + 6,   #  writes them they are read from the snapshot)  + m read and write; Delta zero store elided
 }
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
@@ -377,9 +377,9 @@ def main_ksweep(args):
         adam_ms = sum(b.elapsed_time(c) for _, b, c in ev) / len(ev)
         # one full cycle per round (N = W = 8): theta read+written per batch, Delta read on all batches but the
         # first and written on all but the last, m read+written once; per batch k worker vectors and the one
-        # snapshot its workers share are read, k x (params 4 + bf16 2) and one new snapshot are written
+        # snapshot its workers share are read, k bf16 replicas and one new snapshot are written
         nb = W // k
-        arr_bytes = (8 * nb + 8 * (nb - 1) + 8 + nb * (4 * k + 4) + nb * (6 * k + 4)) * P
+        arr_bytes = (8 * nb + 8 * (nb - 1) + 8 + nb * (4 * k + 4) + nb * (2 * k + 4)) * P
         adam_bytes = ADAMW_BYTES * P * W * inner
         out.append({"k": k, "arrival_ms_per_round": arr_ms, "arrival_gbs": arr_bytes / arr_ms / 1e6,
                     "arrival_frac": arr_bytes / arr_ms / 1e6 / peak, "arrival_bytes_per_param_per_arrival": arr_bytes / P / W,

@@ -26,6 +26,9 @@ struct Worker {
     uint16_t* rep = nullptr;
     uint64_t pull_tick = 0;
     WorkerState state = kNever;
+    // Right after a dispatch the worker's parameters equal its snapshot.  With snapshots in use the
+    // copy into p is not made: readers take the snapshot instead until something writes p.
+    bool p_in_snapshot = false;
 };
 
 uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
@@ -186,10 +189,24 @@ int copy_vec(alsgd_ctx* c, void* dst, const void* src, uint64_t bytes, bool host
 
 // Re-seed target: the worker's parameters and replica, plus (for one worker of the window) the
 // snapshot slot the whole window will share.
-void fill_seed(ArriveArgs& a, uint32_t slot, const Worker& w, float* snapshot) {
-    a.seed_p[slot] = w.p;
+void fill_seed(ArriveArgs& a, uint32_t slot, const Worker& w, float* snapshot, bool have_snapshots) {
+    a.seed_p[slot] = have_snapshots ? nullptr : w.p;     // with snapshots the parameters are read from there
     a.seed_base[slot] = snapshot;
     a.seed_rep[slot] = w.rep;
+}
+
+// Where the worker's current parameters are to be read from.
+const float* params_of(const Worker& w) { return w.p_in_snapshot ? w.base : w.p; }
+
+// Make w.p hold the worker's parameters before handing the pointer out or copying from it.
+int materialize_params(alsgd_ctx* c, Worker& w) {
+    if (!w.p_in_snapshot) return ALSGD_OK;
+    if (cudaMemcpyAsync(w.p, w.base, sizeof(float) * c->P, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) {
+        c->last_cuda = (int)cudaGetLastError();
+        return ALSGD_E_CUDA;
+    }
+    w.p_in_snapshot = false;
+    return ALSGD_OK;
 }
 
 // The slot that is free once the given workers have let go of theirs (-1 when the pseudo-gradient
@@ -214,6 +231,7 @@ void commit_slot(alsgd_ctx* c, const uint32_t* ids, uint32_t k, int s) {
         if (w.slot >= 0) --c->slot_ref[w.slot];
         w.slot = s;
         w.base = c->slot_ptr[s];
+        w.p_in_snapshot = true;
         ++c->slot_ref[s];
     }
 }
@@ -327,6 +345,7 @@ int alsgd_set_worker_params(alsgd_ctx* c, uint32_t worker, const float* src, int
     if (!c || !src) return ALSGD_E_ARG;
     if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
     DeviceGuard g(c->cfg.device);
+    c->workers[worker].p_in_snapshot = false;            // overwritten in full
     return copy_vec(c, c->workers[worker].p, src, sizeof(float) * c->P, !src_is_device);
 }
 
@@ -334,7 +353,7 @@ int alsgd_get_worker_params(alsgd_ctx* c, uint32_t worker, float* dst, int dst_i
     if (!c || !dst) return ALSGD_E_ARG;
     if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
     DeviceGuard g(c->cfg.device);
-    return copy_vec(c, dst, c->workers[worker].p, sizeof(float) * c->P, !dst_is_device);
+    return copy_vec(c, dst, params_of(c->workers[worker]), sizeof(float) * c->P, !dst_is_device);
 }
 
 int alsgd_pull(alsgd_ctx* c, uint32_t worker) {
@@ -347,7 +366,7 @@ int alsgd_pull(alsgd_ctx* c, uint32_t worker) {
     a.n_arr = 0;
     a.n_seed = 1;
     const int slot = pick_slot(c, &worker, 1);
-    fill_seed(a, 0, w, slot >= 0 ? c->slot_ptr[slot] : nullptr);
+    fill_seed(a, 0, w, slot >= 0 ? c->slot_ptr[slot] : nullptr, slot >= 0);
     DeviceGuard g(c->cfg.device);
     ALSGD_CUDA(c, launch_arrive(a, false, false, false, c->lc, c->stream));
     commit_slot(c, &worker, 1, slot);
@@ -371,7 +390,7 @@ int alsgd_inner_adamw(alsgd_ctx* c, uint32_t worker, const float* grads, int gra
         gdev = c->grad_stage;
     }
     AdamArgs a{};
-    a.p = w.p; a.m = w.am; a.v = w.av; a.g = gdev; a.rep = w.rep;
+    a.p = w.p; a.p_src = params_of(w); a.m = w.am; a.v = w.av; a.g = gdev; a.rep = w.rep;
     a.seg_end = c->seg_end; a.seg_decay = c->seg_decay; a.n_seg = c->n_seg;
     a.n = c->P;
     a.b1 = c->cfg.adam_b1; a.b2 = c->cfg.adam_b2;
@@ -381,6 +400,7 @@ int alsgd_inner_adamw(alsgd_ctx* c, uint32_t worker, const float* grads, int gra
     a.bc2 = (float)(1.0 - std::pow((double)a.b2, (double)step));
     a.eps = c->cfg.adam_eps; a.lr = lr; a.wd = c->cfg.adam_wd;
     ALSGD_CUDA(c, launch_adamw(a, c->lc, c->stream));
+    w.p_in_snapshot = false;
     return ALSGD_OK;
 }
 
@@ -470,7 +490,7 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
         for (uint32_t j = 0; j < kk; ++j) {
             const uint32_t src = active[j0 + j];
             const Worker& w = c->workers[ids[src]];
-            a.p[j] = w.p;
+            a.p[j] = params_of(w);
             a.base[j] = w.base;
             a.w[j] = plan[src].weight;
             const bool b = ((plan[src].tick + 1) % N) == 0;          // Algorithm 3's boundary test
@@ -490,7 +510,7 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
         if (any_boundary) a.flags |= kReadM | kWriteM;
         if (reseed && ch + 1 == n_chunks) {               // the final theta exists only in the last pass
             const uint32_t ns = k < (uint32_t)kMaxSeeds ? k : (uint32_t)kMaxSeeds;
-            for (uint32_t s = 0; s < ns; ++s) fill_seed(a, s, c->workers[ids[k - ns + s]], s == 0 ? snapshot : nullptr);
+            for (uint32_t s = 0; s < ns; ++s) fill_seed(a, s, c->workers[ids[k - ns + s]], s == 0 ? snapshot : nullptr, snapshot != nullptr);
             a.n_seed = ns;
             seeded = ns;
             snapshot_written = true;
@@ -520,7 +540,7 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
             ArriveArgs a{};
             a.theta = c->theta; a.n = c->P; a.n_seed = ns;
             for (uint32_t s = 0; s < ns; ++s) {
-                fill_seed(a, s, c->workers[ids[at + s]], snapshot_written ? nullptr : snapshot);
+                fill_seed(a, s, c->workers[ids[at + s]], snapshot_written ? nullptr : snapshot, snapshot != nullptr);
                 snapshot_written = true;
             }
             ALSGD_CUDA(c, launch_arrive(a, false, false, false, c->lc, c->stream));
@@ -588,7 +608,12 @@ int alsgd_state_ptrs(alsgd_ctx* c, alsgd_ptrs* out) {
 int alsgd_worker_state_ptrs(alsgd_ctx* c, uint32_t worker, alsgd_worker_ptrs* out) {
     if (!c || !out) return ALSGD_E_ARG;
     if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
-    const Worker& w = c->workers[worker];
+    Worker& w = c->workers[worker];
+    {
+        DeviceGuard g(c->cfg.device);
+        const int rc = materialize_params(c, w);
+        if (rc != ALSGD_OK) return rc;
+    }
     out->p = w.p; out->base = w.base; out->adam_m = w.am; out->adam_v = w.av; out->replica = w.rep;
     return ALSGD_OK;
 }
@@ -656,6 +681,10 @@ int alsgd_export_state(alsgd_ctx* c, void* host_dst, uint64_t bytes) {
         ALSGD_CUDA(c, cudaMemsetAsync(c->delta, 0, sizeof(float) * c->P, c->stream));
         c->delta_stored = true;
     }
+    for (Worker& w : c->workers) {
+        const int rc = materialize_params(c, w);
+        if (rc != ALSGD_OK) return rc;
+    }
     uint8_t* out = static_cast<uint8_t*>(host_dst);
     ImageHeader h{};
     std::memcpy(h.magic, kMagic, 8);
@@ -700,6 +729,7 @@ int alsgd_import_state(alsgd_ctx* c, const void* host_src, uint64_t bytes) {
         c->workers[w].base = c->slot_ptr[w];
         c->slot_ref[w] = 1u;
     }
+    for (Worker& w : c->workers) w.p_in_snapshot = false;       // the image carries the parameters themselves
     int rc = for_each_slice(c, [&](void* dev, uint64_t n) -> int {
         if (cudaMemcpyAsync(dev, in, n, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return cuda_fail(c, cudaGetLastError());
         in += n;

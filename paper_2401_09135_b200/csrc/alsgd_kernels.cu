@@ -154,7 +154,7 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
 #pragma unroll
                 for (int s = 0; s < kMaxSeeds; ++s) {
                     if (s < (int)a.n_seed) {
-                        st_stream(reinterpret_cast<float4*>(a.seed_p[s]) + i, th[v]);
+                        if (a.seed_p[s]) st_stream(reinterpret_cast<float4*>(a.seed_p[s]) + i, th[v]);
                         if (a.seed_base[s]) st_stream(reinterpret_cast<float4*>(a.seed_base[s]) + i, th[v]);
                         if (a.seed_rep[s]) st_stream(reinterpret_cast<uint2*>(a.seed_rep[s]) + i, packed);
                     }
@@ -183,7 +183,7 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
             if (write_m) a.mom[i] = mm;
         }
         for (uint32_t s = 0; s < a.n_seed; ++s) {
-            a.seed_p[s][i] = th;
+            if (a.seed_p[s]) a.seed_p[s][i] = th;
             if (a.seed_base[s]) a.seed_base[s][i] = th;
             if (a.seed_rep[s]) a.seed_rep[s][i] = (uint16_t)bf16_bits(th);
         }
@@ -259,7 +259,8 @@ template <int V>
 __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ AdamArgs a) {
     const uint64_t nvec = a.n >> 2;
     const uint64_t tile = (uint64_t)kBlock * V;
-    float4* __restrict__ p4 = reinterpret_cast<float4*>(a.p);
+    float4* p4 = reinterpret_cast<float4*>(a.p);
+    const float4* ps4 = reinterpret_cast<const float4*>(a.p_src);
     float4* __restrict__ m4 = reinterpret_cast<float4*>(a.m);
     float4* __restrict__ v4 = reinterpret_cast<float4*>(a.v);
     const float4* __restrict__ g4 = reinterpret_cast<const float4*>(a.g);
@@ -276,7 +277,7 @@ __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ A
             const uint64_t i = t0 + (uint64_t)k * kBlock + threadIdx.x;
             if (i < nvec) {
                 g[k] = ld_stream(g4 + i);
-                p[k] = ld_stream(p4 + i);
+                p[k] = ld_stream(ps4 + i);
                 m[k] = ld_stream(m4 + i);
                 v[k] = ld_stream(v4 + i);
             }
@@ -315,7 +316,7 @@ __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ A
     if (blockIdx.x == 0 && rem0 + threadIdx.x < a.n) {
         const uint64_t i = rem0 + threadIdx.x;
         SegCursor c = seg_find(i, a);
-        float p = a.p[i], m = a.m[i], v = a.v[i];
+        float p = a.p_src[i], m = a.m[i], v = a.v[i];
         adam_element(p, m, v, a.g[i], c.decay != 0, a);
         a.p[i] = p;
         a.m[i] = m;

@@ -26,7 +26,7 @@ struct ArriveArgs {
     float* mom;
     const float* base[kMaxArrivals];  // dispatch snapshots (unused when the pseudo-gradient is against running theta)
     const float* p[kMaxArrivals];     // arriving workers' parameters
-    float* seed_p[kMaxSeeds];
+    float* seed_p[kMaxSeeds];         // may be null (parameters are then read from the snapshot until first written)
     float* seed_base[kMaxSeeds];      // may be null
     uint16_t* seed_rep[kMaxSeeds];    // may be null
     double* gnorm2;                   // scratch: kMaxArrivals accumulators, zeroed by the caller
@@ -44,7 +44,8 @@ struct ArriveArgs {
 };
 
 struct AdamArgs {
-    float* p;
+    float* p;                  // parameters out
+    const float* p_src;        // parameters in (p itself, or the dispatch snapshot right after a dispatch)
     float* m;
     float* v;
     const float* g;

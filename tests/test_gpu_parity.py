@@ -278,6 +278,48 @@ def test_transformer_110m_eight_workers_batch_sweep(k, N):
     pair.close()
 
 
+def test_reseeded_parameters_are_read_from_the_snapshot_until_written():
+    """After a dispatch the library does not store the worker's parameters a second time; every reader
+    (AdamW, an arrival, alsgd_get_worker_params) must still see them.  No device pointer of a worker is
+    requested between the re-seed and the next use, so the deferred copy is never forced."""
+    tensors = synth.ragged_tensors()
+    W = 4
+    pair = Pair(tensors, W, 3, 0.9, 0.7, align=8)
+    P = pair.P
+    pair.set_global(synth.theta0(tensors, pair.offsets, P, SEED + 9))
+    for w in range(W):
+        pair.pull(w)
+    got = torch.empty(P, dtype=torch.float32, device="cuda")
+    life = [0] * W
+
+    def adam(w):
+        life[w] += 1
+        g = synth.zero_padding(synth.normal_vec(P, 1e-2, SEED + 9, synth.STREAM_GRAD, sub=w * 50 + life[w]), tensors, pair.offsets)
+        pair.inner_adamw(w, dev(g), g, life[w], 1e-3)
+
+    def check_params(w, where):
+        pair.ctx.alsgd_get_worker_params(w, got)
+        pair.ctx.alsgd_sync()
+        assert_fp32(f"params[{w}] {where}", pair.fetch(got), pair.orc.p[w])
+
+    adam(0); adam(0); adam(1)
+    pair.arrive([0, 2, 1], reseed=True)          # worker 2 arrives untouched: its pseudo-gradient is exactly zero
+    pair.check_server("first window")
+    for w in (0, 1, 2):
+        check_params(w, "after re-seed")         # equals theta, read through the snapshot
+    adam(0); adam(2)                             # first step after the re-seed reads the shared snapshot
+    check_params(0, "after AdamW")
+    pair.arrive([2], reseed=True)
+    pair.arrive([1, 3], reseed=True)             # 1 never ran a step since its dispatch; 3 never since the start
+    adam(1); adam(3); adam(0)
+    pair.arrive([0, 3, 1, 2], reseed=True)
+    pair.check_server("last window")
+    for w in range(W):
+        check_params(w, "end")
+    pair.check_all("end")
+    pair.close()
+
+
 # --------------------------------------------------------------------------------------------------
 # Host gradients, diagnostics, error paths (all made on the host; nothing here faults the device)
 # --------------------------------------------------------------------------------------------------
