@@ -101,6 +101,7 @@ struct alsgd_ctx {
     uint32_t* seg_decay = nullptr;
     uint32_t n_seg = 0;
     double* gnorm2 = nullptr;
+    double* diag_partial = nullptr;
     unsigned int* nonfinite = nullptr;
     float* theta = nullptr;
     float* mom = nullptr;
@@ -128,12 +129,13 @@ uint64_t carve(alsgd_ctx* c, void* arena, uint64_t P, const alsgd_config& cfg, u
     uint64_t* seg_end = k.take<uint64_t>(n_seg);
     uint32_t* seg_decay = k.take<uint32_t>(n_seg);
     double* gn = k.take<double>(kMaxArrivals);
+    double* gpart = k.take<double>(diag_partial_count(P));
     unsigned int* nf = k.take<unsigned int>(kMaxArrivals);
     float* theta = k.take<float>(P);
     float* mom = k.take<float>(P);
     float* delta = k.take<float>(P);
     if (c) {
-        c->seg_end = seg_end; c->seg_decay = seg_decay; c->gnorm2 = gn; c->nonfinite = nf;
+        c->seg_end = seg_end; c->seg_decay = seg_decay; c->gnorm2 = gn; c->diag_partial = gpart; c->nonfinite = nf;
         c->theta = theta; c->mom = mom; c->delta = delta;
         c->workers.assign(cfg.n_workers, Worker());
         c->slot_ptr.clear();
@@ -479,7 +481,7 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
         const uint32_t kk = (ka - j0 < (uint32_t)kMaxArrivals) ? ka - j0 : (uint32_t)kMaxArrivals;
         ArriveArgs a{};
         a.theta = c->theta; a.delta = c->delta; a.mom = c->mom;
-        a.gnorm2 = c->gnorm2; a.nonfinite = c->nonfinite;
+        a.gnorm2 = c->gnorm2; a.diag_partial = c->diag_partial; a.nonfinite = c->nonfinite;
         a.n = c->P;
         a.n_arr = kk;
         a.beta = c->cfg.beta; a.eps = c->cfg.outer_lr; a.inv_n = c->inv_n; a.cb = c->cb; a.cn = c->cn;
@@ -516,7 +518,6 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
             snapshot_written = true;
         }
         if (diag) {
-            ALSGD_CUDA(c, cudaMemsetAsync(c->gnorm2, 0, sizeof(double) * kMaxArrivals, c->stream));
             ALSGD_CUDA(c, cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * kMaxArrivals, c->stream));
         }
         ALSGD_CUDA(c, launch_arrive(a, current, diag, extended, c->lc, c->stream));

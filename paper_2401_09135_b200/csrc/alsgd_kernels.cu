@@ -189,7 +189,9 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
         }
     }
 
-    // ---- optional diagnostics: one double atomic per block per arrival, one flag per arrival
+    // ---- optional diagnostics: one partial sum per block per arrival, added up in a fixed order by
+    //      diag_reduce_kernel (no atomics: 10^5 blocks adding into a handful of addresses serialise in
+    //      one L2 slice and cost up to 40 % of the pass); one flag per arrival
     if (DIAG && K > 0) {
         __shared__ double warp_sum[kBlock / 32][KK];
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -209,8 +211,24 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
         if ((int)threadIdx.x < K) {
             double s = 0.0;
             for (int w = 0; w < kBlock / 32; ++w) s += warp_sum[w][threadIdx.x];
-            atomicAdd(a.gnorm2 + threadIdx.x, s);
+            a.diag_partial[(uint64_t)blockIdx.x * K + threadIdx.x] = s;
         }
+    }
+}
+
+// Block j adds the per-block partial sums of arrival j in index order.
+__global__ void __launch_bounds__(kBlock) diag_reduce_kernel(const double* __restrict__ partial, uint32_t n_blocks,
+                                                             uint32_t K, double* __restrict__ out) {
+    __shared__ double lane_sum[kBlock];
+    const uint32_t j = blockIdx.x;
+    double s = 0.0;
+    for (uint32_t b = threadIdx.x; b < n_blocks; b += kBlock) s += partial[(uint64_t)b * K + j];
+    lane_sum[threadIdx.x] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int i = 0; i < kBlock; ++i) t += lane_sum[i];
+        out[j] = t;
     }
 }
 
@@ -351,6 +369,7 @@ cudaError_t launch_arrive_k(const ArriveArgs& a, const LaunchCfg& lc, cudaStream
     if (e != cudaSuccess) return e;
     (void)lc;
     kern<<<grid, kBlock, 0, s>>>(a);
+    if (DIAG && K > 0) diag_reduce_kernel<<<K, kBlock, 0, s>>>(a.diag_partial, grid, K, a.gnorm2);
     return cudaGetLastError();
 }
 
@@ -376,6 +395,11 @@ cudaError_t launch_arrive_e(const ArriveArgs& a, bool extended, const LaunchCfg&
 }
 
 }  // namespace
+
+uint64_t diag_partial_count(uint64_t n) {
+    const uint64_t blocks = ((n >> 2) + kBlock - 1) / kBlock + 1;    // one float4 per thread gives the most blocks
+    return blocks * kMaxArrivals;
+}
 
 cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, bool extended, const LaunchCfg& lc, cudaStream_t s) {
     if (a.n == 0) return cudaSuccess;

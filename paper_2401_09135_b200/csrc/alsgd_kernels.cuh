@@ -29,7 +29,8 @@ struct ArriveArgs {
     float* seed_p[kMaxSeeds];         // may be null (parameters are then read from the snapshot until first written)
     float* seed_base[kMaxSeeds];      // may be null
     uint16_t* seed_rep[kMaxSeeds];    // may be null
-    double* gnorm2;                   // scratch: kMaxArrivals accumulators, zeroed by the caller
+    double* gnorm2;                   // out: kMaxArrivals squared norms (written by the reduction that follows the pass)
+    double* diag_partial;             // scratch: one double per block per arrival, diag_partial_count(n) entries
     unsigned int* nonfinite;          // scratch: kMaxArrivals flags, zeroed by the caller
     uint64_t n;                       // elements
     uint32_t n_arr;
@@ -60,6 +61,9 @@ struct AdamArgs {
 struct LaunchCfg {
     int sm_count;
 };
+
+// Entries of ArriveArgs::diag_partial needed for a vector of n elements (any batch size).
+uint64_t diag_partial_count(uint64_t n);
 
 cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, bool extended, const LaunchCfg& lc, cudaStream_t s);
 cudaError_t launch_adamw(const AdamArgs& a, const LaunchCfg& lc, cudaStream_t s);

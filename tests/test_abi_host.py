@@ -93,11 +93,12 @@ def test_arena_bytes_accounts_for_every_buffer():
     P = 22_914_816
     n = C.c_uint64()
     assert L.alsgd_arena_bytes(tab, len(tab), 128, C.byref(_cfg()), C.byref(n)) == 0
-    body = 12 * P + 4 * 18 * P          # theta, m, Delta + 4 x (p, base, adam m, adam v, bf16)
-    assert body <= n.value <= body + 64 * 1024
+    body = 12 * P + 4 * 18 * P          # theta, m, Delta + 4 x (p, snapshot, adam m, adam v, bf16)
+    slack = P // 16 + 64 * 1024         # diagnostics partial sums (one double per 1024 elements per arrival slot) + tables
+    assert body <= n.value <= body + slack
     m = C.c_uint64()
     assert L.alsgd_arena_bytes(tab, len(tab), 128, C.byref(_cfg(pg_base=B.PG_CURRENT, flags=0)), C.byref(m)) == 0
-    assert 12 * P + 4 * 12 * P <= m.value <= 12 * P + 4 * 12 * P + 64 * 1024
+    assert 12 * P + 4 * 12 * P <= m.value <= 12 * P + 4 * 12 * P + slack
     g = C.c_uint64()
     assert L.alsgd_arena_bytes(tab, len(tab), 128, C.byref(_cfg(flags=B.CFG_REPLICA_BF16 | B.CFG_GRAD_STAGING)), C.byref(g)) == 0
     assert g.value - n.value == 4 * P
