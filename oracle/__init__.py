@@ -37,41 +37,45 @@ _u32p = C.POINTER(C.c_uint32)
 _f64p = C.POINTER(C.c_double)
 
 
+def _configure(L):
+    """Declare the argument and result types of every oracle function on a loaded library."""
+    L.orc_bf16_rne.argtypes = [C.c_uint32]
+    L.orc_bf16_rne.restype = C.c_uint16
+    L.orc_cast_bf16.argtypes = [_f32p, _u16p, C.c_uint64, C.c_uint64]
+    L.orc_cast_bf16.restype = None
+    L.orc_inv_n.argtypes = [C.c_uint32]
+    L.orc_inv_n.restype = C.c_float
+    L.orc_boundary_weight.argtypes = [C.c_uint32, C.c_float, C.c_float]
+    L.orc_boundary_weight.restype = C.c_float
+    L.orc_between_weight.argtypes = [C.c_float, C.c_float]
+    L.orc_between_weight.restype = C.c_float
+    L.orc_dn_arrive.argtypes = [_f32p, _f32p, _f32p, _f32p, _f32p, C.c_uint64, C.c_uint64, C.c_uint64,
+                                C.c_uint32, C.c_float, C.c_float, C.c_float, C.c_int, C.c_float,
+                                C.c_float, C.c_int]
+    L.orc_dn_arrive.restype = C.c_int
+    L.orc_pg_norm2.argtypes = [_f32p, _f32p, _f32p, C.c_uint64, C.c_uint64, C.c_int, _u32p]
+    L.orc_pg_norm2.restype = C.c_double
+    L.orc_reseed.argtypes = [_f32p, _f32p, _f32p, _u16p, C.c_uint64, C.c_uint64]
+    L.orc_reseed.restype = None
+    L.orc_adamw.argtypes = [_f32p, _f32p, _f32p, _f32p, _u16p, _u8p, C.c_uint64, C.c_uint64, C.c_uint64,
+                            C.c_float, C.c_float, C.c_float, C.c_float, C.c_float]
+    L.orc_adamw.restype = None
+    L.orc_dylu.argtypes = [_f64p, C.c_uint32, C.c_uint32, _u32p]
+    L.orc_dylu.restype = None
+    L.orc_lr_at.argtypes = [C.c_double, C.c_double, C.c_uint64, C.c_uint64, C.c_uint64]
+    L.orc_lr_at.restype = C.c_double
+    L.orc_poly_weight.argtypes = [C.c_uint64]
+    L.orc_poly_weight.restype = C.c_float
+    L.orc_schedule.argtypes = [C.c_uint32, _f64p, C.c_uint32, _u32p, C.c_double, C.c_uint64, C.c_uint32,
+                               _u32p, _f64p, _u32p]
+    L.orc_schedule.restype = C.c_uint32
+    return L
+
+
 def lib():
     global _lib
     if _lib is None:
-        L = C.CDLL(build())
-        L.orc_bf16_rne.argtypes = [C.c_uint32]
-        L.orc_bf16_rne.restype = C.c_uint16
-        L.orc_cast_bf16.argtypes = [_f32p, _u16p, C.c_uint64, C.c_uint64]
-        L.orc_cast_bf16.restype = None
-        L.orc_inv_n.argtypes = [C.c_uint32]
-        L.orc_inv_n.restype = C.c_float
-        L.orc_boundary_weight.argtypes = [C.c_uint32, C.c_float, C.c_float]
-        L.orc_boundary_weight.restype = C.c_float
-        L.orc_between_weight.argtypes = [C.c_float, C.c_float]
-        L.orc_between_weight.restype = C.c_float
-        L.orc_dn_arrive.argtypes = [_f32p, _f32p, _f32p, _f32p, _f32p, C.c_uint64, C.c_uint64, C.c_uint64,
-                                    C.c_uint32, C.c_float, C.c_float, C.c_float, C.c_int, C.c_float,
-                                    C.c_float, C.c_int]
-        L.orc_dn_arrive.restype = C.c_int
-        L.orc_pg_norm2.argtypes = [_f32p, _f32p, _f32p, C.c_uint64, C.c_uint64, C.c_int, _u32p]
-        L.orc_pg_norm2.restype = C.c_double
-        L.orc_reseed.argtypes = [_f32p, _f32p, _f32p, _u16p, C.c_uint64, C.c_uint64]
-        L.orc_reseed.restype = None
-        L.orc_adamw.argtypes = [_f32p, _f32p, _f32p, _f32p, _u16p, _u8p, C.c_uint64, C.c_uint64, C.c_uint64,
-                                C.c_float, C.c_float, C.c_float, C.c_float, C.c_float]
-        L.orc_adamw.restype = None
-        L.orc_dylu.argtypes = [_f64p, C.c_uint32, C.c_uint32, _u32p]
-        L.orc_dylu.restype = None
-        L.orc_lr_at.argtypes = [C.c_double, C.c_double, C.c_uint64, C.c_uint64, C.c_uint64]
-        L.orc_lr_at.restype = C.c_double
-        L.orc_poly_weight.argtypes = [C.c_uint64]
-        L.orc_poly_weight.restype = C.c_float
-        L.orc_schedule.argtypes = [C.c_uint32, _f64p, C.c_uint32, _u32p, C.c_double, C.c_uint64, C.c_uint32,
-                                   _u32p, _f64p, _u32p]
-        L.orc_schedule.restype = C.c_uint32
-        _lib = L
+        _lib = _configure(C.CDLL(build()))
     return _lib
 
 

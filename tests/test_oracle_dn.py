@@ -196,6 +196,11 @@ def test_current_mode_uses_running_theta():
     # g = theta - p = (0.5, -0.5); theta -= 0.5 * g/4
     np.testing.assert_array_equal(D, [0.5, -0.5])
     np.testing.assert_array_equal(theta, [1.0 - 0.0625, 2.0 + 0.0625])
+    # a dispatch snapshot, if one is handed in, plays no part in this mode
+    theta2, m2, D2 = np.array([1.0, 2.0], np.float32), np.zeros(2, np.float32), np.zeros(2, np.float32)
+    oracle.dn_arrive(theta2, m2, D2, np.array([99.0, -99.0], np.float32), p, 0, 4, 0.5, 0.5, 0.0, pg_current=True)
+    np.testing.assert_array_equal(D2, [0.5, -0.5])
+    np.testing.assert_array_equal(theta2, theta)
 
 
 def test_brute_force_batch_orders_tiny():
