@@ -40,9 +40,9 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter from the committed ncu captures
 # (profiles/), valid only for the kernel source they were taken from.
 NCU_TRAFFIC = {
-    "src_sha256": "d9891adf4afa45d7f7b9ad854dba32674240bfbd312755ef4cb7a2d985ffb255",
-    "adamw_bytes_per_param": 28.88,     # profiles/adamw_kernel_flat48M.md (P = 50.3M, scaled by P)
-    "arrive_bytes_per_param": 32.86,    # profiles/arrive_kernel_flat48M.md, K = 1 cycle average
+    "src_sha256": "8e2b88c8f7fa790061e2ca71d44678ac12f83c85dc806f6c7ce70aa371c2abe3",
+    "adamw_bytes_per_param": 28.90,     # profiles/adamw_kernel_flat48M.md (P = 50.3M, scaled by P)
+    "arrive_bytes_per_param": 28.90,    # profiles/arrive_kernel_flat48M.md, K = 1 cycle average
 }
 
 

@@ -3,9 +3,9 @@ but only ~2.4 GB on the device in total.
 
     python -m paper_2401_09135_b200.profile_case [--elems N]
 
-Launch order: 2 pulls, 3 AdamW steps on worker 0, 3 on worker 1, then single arrivals with fused
-re-seed through one Delayed-Nesterov cycle of N = 4 (first / middle / middle / boundary), then one
-batch of two.
+Launch order: 2 pulls, 3 AdamW steps on worker 0, 3 on worker 1, then four times (one AdamW step,
+one single arrival with fused re-seed) through one Delayed-Nesterov cycle of N = 4 (first / middle /
+middle / boundary), then one AdamW step per worker and one batch of two: 19 launches.
 """
 import argparse
 
@@ -31,8 +31,14 @@ def main():
     for w in range(2):
         for s in range(1, 4):
             ctx.alsgd_inner_adamw(w, g, s, 1e-3)
+    step = [3, 3]
     for w in (0, 1, 0, 1):
+        step[w] += 1
+        ctx.alsgd_inner_adamw(w, g, step[w], 1e-3)
         ctx.alsgd_arrive([w], B.ARRIVE_RESEED, want_info=False)
+    for w in range(2):
+        step[w] += 1
+        ctx.alsgd_inner_adamw(w, g, step[w], 1e-3)
     ctx.alsgd_arrive([0, 1], B.ARRIVE_RESEED, want_info=False)
     ctx.alsgd_sync()
     print(f"profile case done: P={ctx.P}, t={ctx.alsgd_counters()[0]}")
