@@ -237,6 +237,12 @@ int alsgd_last_cuda_error(alsgd_ctx* ctx);
  * speeds: host, n positive values (steps per second).  steps_out: host, n entries. */
 int alsgd_dylu_steps(const double* speeds, uint32_t n, uint32_t H, uint32_t* steps_out);
 
+/* Data-shard sampling, Eq. 2: probs_i proportional to max(sizes_i / sum sizes - learned_i / sum learned, 0),
+ * learned_i = data points already learned from shard i, so that under-sampled shards are preferred.  While
+ * nothing has been learned the learned share counts as 0; if no shard is under-sampled the size shares are
+ * returned.  sizes (> 0), learned (>= 0), probs_out: host, n entries.  The draw itself is the caller's. */
+int alsgd_shard_probs(const double* sizes, const double* learned, uint32_t n, double* probs_out);
+
 typedef struct alsgd_lr_sched {
     double eta_max, eta_min;
     uint64_t t_warmup, T;

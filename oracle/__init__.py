@@ -66,6 +66,8 @@ def _configure(L):
     L.orc_lr_at.restype = C.c_double
     L.orc_poly_weight.argtypes = [C.c_uint64]
     L.orc_poly_weight.restype = C.c_float
+    L.orc_shard_probs.argtypes = [_f64p, _f64p, C.c_uint32, _f64p]
+    L.orc_shard_probs.restype = None
     L.orc_schedule.argtypes = [C.c_uint32, _f64p, C.c_uint32, _u32p, C.c_double, C.c_uint64, C.c_uint32,
                                _u32p, _f64p, _u32p]
     L.orc_schedule.restype = C.c_uint32
@@ -149,6 +151,15 @@ def lr_at(eta_max, eta_min, t_warmup, T, t) -> float:
 
 def poly_weight(staleness: int) -> float:
     return float(lib().orc_poly_weight(int(staleness)))
+
+
+def shard_probs(sizes, learned):
+    """Eq. 2: sampling probability of every data shard."""
+    s = np.ascontiguousarray(sizes, dtype=np.float64)
+    l = np.ascontiguousarray(learned, dtype=np.float64)
+    out = np.zeros(s.shape[0], dtype=np.float64)
+    lib().orc_shard_probs(_p(s, _f64p), _p(l, _f64p), s.shape[0], _p(out, _f64p))
+    return [float(x) for x in out]
 
 
 def schedule(durations, local_updates, tau_grace, t_max, max_arrivals):

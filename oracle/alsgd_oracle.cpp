@@ -17,6 +17,7 @@
 //   orc_dylu        Eq. 6 values for speeds 1:1.5:2:3, H = 50.
 //   orc_lr_at       Eq. 3 end points and clamps.
 //   orc_schedule    Algorithm 2 + Algorithm 5 on hand timelines (Fig. 3 description).
+//   orc_shard_probs Eq. 2 hand values, normalisation, start-up and balanced special cases.
 //   orc_poly_weight, weight / dc_lambda / buffered arguments of orc_dn_arrive: formulas of Section 4
 //                   ("Existing Fixes"): hand cases, zero-drift and homogeneity properties, buffered
 //                   N = 1 == Eq. 4, buffered == Delayed Nesterov at cycle ends.
@@ -207,6 +208,25 @@ double orc_lr_at(double eta_max, double eta_min, uint64_t t_warmup, uint64_t T, 
     if (ratio > 1.0) ratio = 1.0;
     const double pi = 3.14159265358979323846;
     return eta_min + 0.5 * (eta_max - eta_min) * (1.0 + std::cos(ratio * pi));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. 2, data-shard sampling: p_i proportional to max(|D_i| / sum|D_j| - n_i / sum n_j, 0), with n_i the
+// number of data points already learned from shard i.  Before anything was learned (sum n = 0) the
+// learned share counts as zero; if no shard is under-sampled (all terms zero) the size shares are used.
+// ---------------------------------------------------------------------------------------------
+void orc_shard_probs(const double* sizes, const double* learned, uint32_t n, double* probs) {
+    double total_size = 0.0, total_learned = 0.0;
+    for (uint32_t i = 0; i < n; ++i) { total_size += sizes[i]; total_learned += learned[i]; }
+    double norm = 0.0;
+    for (uint32_t i = 0; i < n; ++i) {
+        const double size_share = sizes[i] / total_size;
+        const double learned_share = total_learned > 0.0 ? learned[i] / total_learned : 0.0;
+        const double gap = size_share - learned_share;
+        probs[i] = gap > 0.0 ? gap : 0.0;
+        norm += probs[i];
+    }
+    for (uint32_t i = 0; i < n; ++i) probs[i] = norm > 0.0 ? probs[i] / norm : sizes[i] / total_size;
 }
 
 // Staleness weight of "Async. DiLoCo + Poly": (1 + staleness)^(-0.5), rounded to binary32.

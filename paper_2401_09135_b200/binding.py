@@ -85,6 +85,7 @@ SIGNATURES = {
     "alsgd_sync": (C.c_int, [_vp]),
     "alsgd_last_cuda_error": (C.c_int, [_vp]),
     "alsgd_dylu_steps": (C.c_int, [_f64p, C.c_uint32, C.c_uint32, _u32p]),
+    "alsgd_shard_probs": (C.c_int, [_f64p, _f64p, C.c_uint32, _f64p]),
     "alsgd_lr_at": (C.c_int, [C.POINTER(LrSched), C.c_uint64, _f64p]),
     "alsgd_sched_create": (C.c_int, [C.POINTER(_vp), C.c_uint32, C.c_double, C.c_uint64]),
     "alsgd_sched_destroy": (C.c_int, [_vp]),
@@ -156,6 +157,15 @@ def alsgd_dylu_steps(speeds, H):
     out = (C.c_uint32 * len(speeds))()
     _check(lib().alsgd_dylu_steps(sp, len(speeds), int(H), out), "alsgd_dylu_steps")
     return [int(x) for x in out]
+
+
+def alsgd_shard_probs(sizes, learned):
+    n = len(sizes)
+    s = (C.c_double * n)(*[float(x) for x in sizes])
+    l = (C.c_double * n)(*[float(x) for x in learned])
+    out = (C.c_double * n)()
+    _check(lib().alsgd_shard_probs(s, l, n, out), "alsgd_shard_probs")
+    return [float(x) for x in out]
 
 
 def alsgd_lr_at(eta_max, eta_min, t_warmup, T, t):

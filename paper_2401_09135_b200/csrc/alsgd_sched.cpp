@@ -45,6 +45,25 @@ int alsgd_dylu_steps(const double* speeds, uint32_t n, uint32_t H, uint32_t* ste
     return ALSGD_OK;
 }
 
+int alsgd_shard_probs(const double* sizes, const double* learned, uint32_t n, double* probs_out) {
+    if (!sizes || !learned || !probs_out || n == 0) return ALSGD_E_ARG;
+    double size_sum = 0.0, learned_sum = 0.0;
+    for (uint32_t i = 0; i < n; ++i) {
+        if (!(sizes[i] > 0.0) || !std::isfinite(sizes[i]) || !(learned[i] >= 0.0) || !std::isfinite(learned[i])) return ALSGD_E_ARG;
+        size_sum += sizes[i];
+        learned_sum += learned[i];
+    }
+    double total = 0.0;
+    for (uint32_t i = 0; i < n; ++i) {
+        const double due = sizes[i] / size_sum;                                   // the shard's share of the data
+        const double had = learned_sum > 0.0 ? learned[i] / learned_sum : 0.0;    // its share of the progress so far
+        probs_out[i] = std::max(due - had, 0.0);
+        total += probs_out[i];
+    }
+    for (uint32_t i = 0; i < n; ++i) probs_out[i] = total > 0.0 ? probs_out[i] / total : sizes[i] / size_sum;
+    return ALSGD_OK;
+}
+
 int alsgd_lr_at(const alsgd_lr_sched* s, uint64_t t, double* lr_out) {
     if (!s || !lr_out) return ALSGD_E_ARG;
     if (!(s->eta_max >= 0.0) || !(s->eta_min >= 0.0)) return ALSGD_E_ARG;

@@ -160,6 +160,20 @@ def test_dylu_matches_oracle():
     assert L.alsgd_dylu_steps((C.c_double * 2)(1.0, 2.0), 2, 0, out) == B.E_ARG
 
 
+def test_shard_probs_match_oracle():
+    r = np.random.default_rng(5)
+    for _ in range(200):
+        n = int(r.integers(1, 12))
+        sizes = list(r.uniform(1, 100, n))
+        learned = list(r.uniform(0, 50, n)) if r.integers(0, 4) else [0.0] * n
+        assert B.alsgd_shard_probs(sizes, learned) == oracle.shard_probs(sizes, learned)
+    assert B.alsgd_shard_probs([1, 3], [5, 15]) == [0.25, 0.75]
+    L = B.lib()
+    out = (C.c_double * 2)()
+    assert L.alsgd_shard_probs((C.c_double * 2)(1.0, 0.0), (C.c_double * 2)(0.0, 0.0), 2, out) == B.E_ARG
+    assert L.alsgd_shard_probs((C.c_double * 2)(1.0, 1.0), (C.c_double * 2)(-1.0, 0.0), 2, out) == B.E_ARG
+
+
 def test_lr_schedule_matches_oracle():
     for (emax, emin, tw, T) in [(0.1, 1e-6, 1000, 88000), (1e-3, 0.0, 0, 100), (0.5, 0.01, 10, 10), (0.5, 0.01, 50, 20)]:
         for t in list(range(0, 130)) + [999, 1000, 1001, 44500, 87999, 88000, 88001, 10**7]:

@@ -176,6 +176,26 @@ def test_lr_schedule_endpoints_and_clamps():
     assert oracle.lr_at(emax, emin, 0, T, 0) == pytest.approx(emax, rel=1e-12)         # no warm-up
 
 
+def test_shard_sampling_eq2():
+    # sizes 1:1:2 -> shares .25 .25 .5 ; learned 10:30:60 -> shares .1 .3 .6 ; gaps .15, <0, <0 -> only shard 0
+    assert oracle.shard_probs([1, 1, 2], [10, 30, 60]) == [1.0, 0.0, 0.0]
+    # learned 40:10:50 -> .4 .1 .5 ; gaps <0, .15, 0 -> only shard 1
+    assert oracle.shard_probs([1, 1, 2], [40, 10, 50]) == [0.0, 1.0, 0.0]
+    # learned 0:25:75 -> 0 .25 .75 ; gaps .25, 0, <0
+    assert oracle.shard_probs([1, 1, 2], [0, 25, 75]) == [1.0, 0.0, 0.0]
+    # two under-sampled shards share in proportion to their gaps: sizes equal, learned 1:2:5 -> gaps 5/24, 2/24, <0
+    p = oracle.shard_probs([1, 1, 1], [1, 2, 5])
+    assert p[2] == 0.0 and abs(p[0] - 5 / 7) < 1e-12 and abs(p[1] - 2 / 7) < 1e-12
+    # nothing learned yet: proportional to shard size; perfectly balanced: also the size shares
+    assert oracle.shard_probs([1, 3], [0, 0]) == [0.25, 0.75]
+    assert oracle.shard_probs([1, 3], [5, 15]) == [0.25, 0.75]
+    r = np.random.default_rng(0)
+    for _ in range(50):
+        n = int(r.integers(1, 9))
+        p = oracle.shard_probs(r.uniform(1, 10, n), r.uniform(0, 10, n))
+        assert abs(sum(p) - 1) < 1e-12 and min(p) >= 0
+
+
 def test_poly_weight():
     assert oracle.poly_weight(0) == 1.0
     assert oracle.poly_weight(3) == 0.5

@@ -27,7 +27,7 @@ ADAM_PINS = [misc.test_adamw_hand_case, misc.test_adamw_first_step_is_sign_step_
              misc.test_adamw_constant_gradient_keeps_sign_stepping, misc.test_adamw_zero_gradient_is_pure_decoupled_decay,
              misc.test_adamw_against_library_adamw_in_double]
 BF16_PINS = [misc.test_bf16_named_values, misc.test_bf16_every_high_half_at_the_critical_low_halves, misc.test_reseed_copies_and_casts]
-HOST_PINS = [misc.test_dylu_values, misc.test_lr_schedule_endpoints_and_clamps, misc.test_poly_weight,
+HOST_PINS = [misc.test_shard_sampling_eq2, misc.test_dylu_values, misc.test_lr_schedule_endpoints_and_clamps, misc.test_poly_weight,
              misc.test_schedule_grace_window_timeline, misc.test_schedule_equal_speeds_behave_synchronously,
              misc.test_schedule_zero_grace_distinct_times_gives_singletons_in_time_order,
              misc.test_schedule_stops_at_t_max_local_updates]
@@ -69,6 +69,9 @@ MUTANTS = [
     ("grace test strict", "completed_time[w] - tau_sync <= tau_grace", "completed_time[w] - tau_sync < tau_grace", None, HOST_PINS),
     ("restart without the grace period", "const double restart = tau_sync + tau_grace;", "const double restart = tau_sync;", None, HOST_PINS),
     ("t_local not counted", "t_local += local_updates[w];", "t_local += 0;", None, HOST_PINS),
+    ("shard gap sign", "const double gap = size_share - learned_share;", "const double gap = learned_share - size_share;", None, HOST_PINS),
+    ("shard gap not clipped at zero", "probs[i] = gap > 0.0 ? gap : 0.0;", "probs[i] = gap > 0.0 ? gap : -gap;", None, HOST_PINS),
+    ("shard probabilities not normalised", "probs[i] = norm > 0.0 ? probs[i] / norm : sizes[i] / total_size;", "probs[i] = norm > 0.0 ? probs[i] : sizes[i] / total_size;", None, HOST_PINS),
     ("Poly exponent", "std::pow(1.0 + (double)staleness, -0.5)", "std::pow(1.0 + (double)staleness, -1.0)", None, VAR_PINS + HOST_PINS),
     ("delay compensation drift sign", "const float drift = theta[i] - start;", "const float drift = start - theta[i];", None, VAR_PINS),
     ("delay compensation with g, not g*g", "(dc_lambda * (g * g))", "(dc_lambda * g)", None, VAR_PINS),
