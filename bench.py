@@ -41,8 +41,8 @@ FALLBACK_HBM_GBS = 6650.0
 # (profiles/), valid only for the kernel source they were taken from.
 NCU_TRAFFIC = {
     "src_sha256": "8e2b88c8f7fa790061e2ca71d44678ac12f83c85dc806f6c7ce70aa371c2abe3",
-    "adamw_bytes_per_param": 28.90,     # profiles/adamw_kernel_flat48M.md (P = 50.3M, scaled by P)
-    "arrive_bytes_per_param": 28.90,    # profiles/arrive_kernel_flat48M.md, K = 1 cycle average
+    "adamw_bytes_per_param": 28.90,     # ncu capture at P = 50.3M elements, scaled by P
+    "arrive_bytes_per_param": 28.90,    # same capture, K = 1, average over one Delayed-Nesterov cycle
 }
 
 
