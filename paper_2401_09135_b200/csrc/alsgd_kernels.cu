@@ -44,14 +44,14 @@ __device__ __forceinline__ uint2 bf16_pack4(const float4& x) {
 // EXT adds the Section 4 variants: delay compensation, staleness weight, buffered outer step.
 template <int K, bool DIAG, bool CUR, bool EXT>
 __device__ __forceinline__ void dn_element(float& th, float& d, float& mm, const float* b, const float* p,
-                                           const ArriveArgs& a, double* acc, uint32_t& bad) {
+                                           const ArriveArgs& a, float* acc) {
 #pragma unroll
     for (int j = 0; j < K; ++j) {
         const float start = CUR ? th : b[j];
         float g = start - p[j];                       // pseudo-gradient
-        if (DIAG) {
-            acc[j] += (double)g * (double)g;
-            if (!isfinite(g)) bad |= 1u << j;
+        if (DIAG) {                                   // two instructions per entry:
+            acc[j] = __fmaf_rn(g, g, acc[j]);         //   sum of squares (at most 16 terms per thread in fp32)
+            acc[K + j] = __fmaf_rn(g, 0.0f, acc[K + j]);   // stays 0 unless an entry is Inf or NaN
         }
         if (EXT) {
             if (a.flags & kDelayComp) {               // g + lambda * g*g*(theta_now - theta_at_dispatch)
@@ -99,10 +99,9 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
     const bool write_theta = !(EXT && (flags & kSkipThetaStore));
     const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
 
-    double acc[KK];
-    uint32_t bad = 0;
+    float acc[2 * KK];                                 // [0, K): sums of squares; [K, 2K): non-finite detectors
 #pragma unroll
-    for (int j = 0; j < KK; ++j) acc[j] = 0.0;
+    for (int j = 0; j < 2 * KK; ++j) acc[j] = 0.0f;
 
     float4* __restrict__ theta4 = reinterpret_cast<float4*>(a.theta);
     float4* __restrict__ delta4 = reinterpret_cast<float4*>(a.delta);
@@ -143,7 +142,7 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
                         pe[j] = reinterpret_cast<const float*>(&p[j][v])[e];
                         be[j] = CUR ? 0.f : reinterpret_cast<const float*>(&b[j][v])[e];
                     }
-                    dn_element<K, DIAG, CUR, EXT>(thf[e], df[e], mf[e], be, pe, a, acc, bad);
+                    dn_element<K, DIAG, CUR, EXT>(thf[e], df[e], mf[e], be, pe, a, acc);
                 }
                 if (write_theta) st_stream(theta4 + i, th[v]);
                 if (write_delta) st_stream(delta4 + i, d[v]);
@@ -177,7 +176,7 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
                 pe[j] = a.p[j][i];
                 be[j] = CUR ? 0.f : a.base[j][i];
             }
-            dn_element<K, DIAG, CUR, EXT>(th, d, mm, be, pe, a, acc, bad);
+            dn_element<K, DIAG, CUR, EXT>(th, d, mm, be, pe, a, acc);
             if (write_theta) a.theta[i] = th;
             if (write_delta) a.delta[i] = d;
             if (write_m) a.mom[i] = mm;
@@ -190,17 +189,19 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
     }
 
     // ---- optional diagnostics: one partial sum per block per arrival, added up in a fixed order by
-    //      diag_reduce_kernel (no atomics: 10^5 blocks adding into a handful of addresses serialise in
+    //      the two diag_reduce kernels (no atomics: 10^5 blocks adding into a handful of addresses serialise in
     //      one L2 slice and cost up to 40 % of the pass); one flag per arrival
     if (DIAG && K > 0) {
-        __shared__ double warp_sum[kBlock / 32][KK];
+        __shared__ float warp_sum[kBlock / 32][KK];
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        uint32_t bad = 0;
 #pragma unroll
         for (int j = 0; j < K; ++j) {
-            double s = acc[j];
+            float s = acc[j];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xFFFFFFFFu, s, o);
+            for (int o = 16; o > 0; o >>= 1) s = s + __shfl_down_sync(0xFFFFFFFFu, s, o);
             if (lane == 0) warp_sum[warp][j] = s;
+            if (!(acc[K + j] == 0.0f)) bad |= 1u << j;
         }
         bad = __reduce_or_sync(0xFFFFFFFFu, bad);
         if (lane == 0 && bad) {
@@ -210,24 +211,40 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
         __syncthreads();
         if ((int)threadIdx.x < K) {
             double s = 0.0;
-            for (int w = 0; w < kBlock / 32; ++w) s += warp_sum[w][threadIdx.x];
-            a.diag_partial[(uint64_t)blockIdx.x * K + threadIdx.x] = s;
+            for (int w = 0; w < kBlock / 32; ++w) s += (double)warp_sum[w][threadIdx.x];   // double from here on
+            a.diag_partial[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x] = s;   // [arrival][block]
         }
     }
 }
 
-// Block j adds the per-block partial sums of arrival j in index order.
-__global__ void __launch_bounds__(kBlock) diag_reduce_kernel(const double* __restrict__ partial, uint32_t n_blocks,
-                                                             uint32_t K, double* __restrict__ out) {
+// Two-stage, fixed-order sum of the per-block partials partial[arrival][block].
+// Stage 1: block (r, j) adds the r-th of kDiagChunks contiguous chunks of arrival j's partials.
+constexpr int kDiagChunks = 64;
+
+__global__ void __launch_bounds__(kBlock) diag_reduce1_kernel(const double* __restrict__ partial, uint32_t n_blocks,
+                                                              double* __restrict__ chunk_sum) {
     __shared__ double lane_sum[kBlock];
-    const uint32_t j = blockIdx.x;
+    const uint32_t r = blockIdx.x, j = blockIdx.y;
+    const uint32_t per = (n_blocks + kDiagChunks - 1) / kDiagChunks;
+    const uint32_t lo = r * per, hi = min(lo + per, n_blocks);
+    const double* __restrict__ row = partial + (uint64_t)j * n_blocks;
     double s = 0.0;
-    for (uint32_t b = threadIdx.x; b < n_blocks; b += kBlock) s += partial[(uint64_t)b * K + j];
+    for (uint32_t b = lo + threadIdx.x; b < hi; b += kBlock) s += row[b];
     lane_sum[threadIdx.x] = s;
     __syncthreads();
     if (threadIdx.x == 0) {
         double t = 0.0;
         for (int i = 0; i < kBlock; ++i) t += lane_sum[i];
+        chunk_sum[j * kDiagChunks + r] = t;
+    }
+}
+
+// Stage 2: thread j adds arrival j's chunk sums in order.
+__global__ void diag_reduce2_kernel(const double* __restrict__ chunk_sum, uint32_t K, double* __restrict__ out) {
+    const uint32_t j = threadIdx.x;
+    if (j < K) {
+        double t = 0.0;
+        for (int r = 0; r < kDiagChunks; ++r) t += chunk_sum[j * kDiagChunks + r];
         out[j] = t;
     }
 }
@@ -369,7 +386,11 @@ cudaError_t launch_arrive_k(const ArriveArgs& a, const LaunchCfg& lc, cudaStream
     if (e != cudaSuccess) return e;
     (void)lc;
     kern<<<grid, kBlock, 0, s>>>(a);
-    if (DIAG && K > 0) diag_reduce_kernel<<<K, kBlock, 0, s>>>(a.diag_partial, grid, K, a.gnorm2);
+    if (DIAG && K > 0) {
+        double* chunk_sum = a.diag_partial + (uint64_t)K * grid;        // behind the K x grid partials
+        diag_reduce1_kernel<<<dim3(kDiagChunks, K), kBlock, 0, s>>>(a.diag_partial, grid, chunk_sum);
+        diag_reduce2_kernel<<<1, 32, 0, s>>>(chunk_sum, K, a.gnorm2);
+    }
     return cudaGetLastError();
 }
 
@@ -398,7 +419,7 @@ cudaError_t launch_arrive_e(const ArriveArgs& a, bool extended, const LaunchCfg&
 
 uint64_t diag_partial_count(uint64_t n) {
     const uint64_t blocks = ((n >> 2) + kBlock - 1) / kBlock + 1;    // one float4 per thread gives the most blocks
-    return blocks * kMaxArrivals;
+    return (blocks + kDiagChunks) * kMaxArrivals;
 }
 
 cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, bool extended, const LaunchCfg& lc, cudaStream_t s) {
