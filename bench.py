@@ -281,6 +281,21 @@ def main_ours(args, rank, world, local_rank):
     h2d = sum(steps[w] for w in e2e_seq) * 4 * P / len(e2e_seq)
     d2h = 4 * P
 
+    # ---- the same AdamW step fed bf16 gradients (28 B/param), reported beside the fp32 figures
+    g16 = [g.to(torch.bfloat16) for g in gpool]
+    for i in range(3):
+        life[0] += 1
+        ctx.alsgd_inner_adamw_bf16(0, g16[i % G], life[0], 1e-3)
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b0.record()
+    for i in range(20):
+        life[0] += 1
+        ctx.alsgd_inner_adamw_bf16(0, g16[i % G], life[0], 1e-3)
+    b1.record()
+    torch.cuda.synchronize()
+    adam16_ms = b0.elapsed_time(b1) / 20
+    del g16
+
     from paper_2401_09135_b200 import shard
     ms, e2e_ms, adam_avg_ms, arr_avg_ms = shard.max_over_ranks(
         [ms, e2e_ms, adam_ms / adam_launches, arr_ms / arr_launches], device="cuda")
@@ -320,6 +335,8 @@ def main_ours(args, rank, world, local_rank):
                                 "traffic": arr_traffic, "bytes_per_param": arr_bytes, "launches": arr_launches,
                                 "avg_ms": arr_avg_ms},
             "params_per_s": {"adamw": P / (adam_avg_ms * 1e-3), "dn_arrival_reseed": P / (arr_avg_ms * 1e-3)},
+            "adamw_bf16_grads": {"avg_ms": adam16_ms, "bytes_per_param": 28, "achieved": 28 * P / (adam16_ms * 1e-3) / 1e9,
+                                 "unit": "GB/s", "launches": 20, "note": "extra; not part of the timed steps"},
         }
         if world == 1 and not args.no_cpu_baseline:
             import oracle

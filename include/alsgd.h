@@ -132,6 +132,12 @@ int alsgd_pull(alsgd_ctx* ctx, uint32_t worker);
 int alsgd_inner_adamw(alsgd_ctx* ctx, uint32_t worker, const float* grads, int grads_is_device,
                       uint64_t step, float lr);
 
+/* The same step with gradients stored as bf16 bit patterns (widened exactly to fp32 before use), as a
+ * mixed-precision backward pass produces them: 28 instead of 30 bytes per parameter on the device and half the
+ * host-to-device traffic.  The paper states no gradient precision; this is an option beside the fp32 call. */
+int alsgd_inner_adamw_bf16(alsgd_ctx* ctx, uint32_t worker, const uint16_t* grads, int grads_is_device,
+                           uint64_t step, float lr);
+
 #define ALSGD_ARRIVE_RESEED 1u    /* re-dispatch all k workers with the final theta (Algorithm 2, the branch taken when get_worker() finds nobody) */
 #define ALSGD_ARRIVE_NORM 2u      /* report the squared norm of each pseudo-gradient */
 #define ALSGD_ARRIVE_NANCHECK 4u  /* report whether each pseudo-gradient has a non-finite entry */

@@ -74,6 +74,7 @@ SIGNATURES = {
     "alsgd_get_worker_params": (C.c_int, [_vp, C.c_uint32, _vp, C.c_int]),
     "alsgd_pull": (C.c_int, [_vp, C.c_uint32]),
     "alsgd_inner_adamw": (C.c_int, [_vp, C.c_uint32, _vp, C.c_int, C.c_uint64, C.c_float]),
+    "alsgd_inner_adamw_bf16": (C.c_int, [_vp, C.c_uint32, _vp, C.c_int, C.c_uint64, C.c_float]),
     "alsgd_arrive": (C.c_int, [_vp, _u32p, C.c_uint32, C.c_uint32, C.POINTER(ArrivalInfo)]),
     "alsgd_arrive_ex": (C.c_int, [_vp, _u32p, C.c_uint32, C.c_uint32, C.POINTER(ArriveOpts), C.POINTER(ArrivalInfo)]),
     "alsgd_counters": (C.c_int, [_vp, _u64p, _u32p]),
@@ -307,6 +308,12 @@ class Context:
         return [{"worker": int(i.worker), "tick": int(i.tick), "staleness": int(i.staleness),
                  "boundary": bool(i.boundary), "gnorm2": float(i.gnorm2), "nonfinite": int(i.nonfinite),
                  "dropped": bool(i.dropped)} for i in info[:k]]
+
+    def alsgd_inner_adamw_bf16(self, w, grads, step, lr):
+        """grads: contiguous torch tensor of P bf16 (or int16 bit patterns), on the device or pinned on the host."""
+        assert grads.is_contiguous() and grads.numel() == self.P and grads.element_size() == 2
+        _check(lib().alsgd_inner_adamw_bf16(self._h, int(w), grads.data_ptr(), int(grads.is_cuda), int(step), float(lr)),
+               "alsgd_inner_adamw_bf16", self._h)
 
     def alsgd_arrive(self, worker_ids, flags=ARRIVE_RESEED, want_info=True):
         k = len(worker_ids)

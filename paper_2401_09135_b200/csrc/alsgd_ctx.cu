@@ -377,8 +377,11 @@ int alsgd_pull(alsgd_ctx* c, uint32_t worker) {
     return ALSGD_OK;
 }
 
-int alsgd_inner_adamw(alsgd_ctx* c, uint32_t worker, const float* grads, int grads_is_device,
-                      uint64_t step, float lr) {
+}  // extern "C"
+
+namespace {
+
+int adamw_impl(alsgd_ctx* c, uint32_t worker, const void* grads, bool bf16, int grads_is_device, uint64_t step, float lr) {
     if (!c || !grads || step == 0) return ALSGD_E_ARG;
     if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
     Worker& w = c->workers[worker];
@@ -386,13 +389,16 @@ int alsgd_inner_adamw(alsgd_ctx* c, uint32_t worker, const float* grads, int gra
     if (!grads_is_device && !c->grad_stage) return ALSGD_E_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(grads) % 16) return ALSGD_E_ARG;
     DeviceGuard g(c->cfg.device);
-    const float* gdev = grads;
+    const void* gdev = grads;
     if (!grads_is_device) {
-        ALSGD_CUDA(c, cudaMemcpyAsync(c->grad_stage, grads, sizeof(float) * c->P, cudaMemcpyHostToDevice, c->stream));
+        const uint64_t bytes = (bf16 ? sizeof(uint16_t) : sizeof(float)) * c->P;
+        ALSGD_CUDA(c, cudaMemcpyAsync(c->grad_stage, grads, bytes, cudaMemcpyHostToDevice, c->stream));
         gdev = c->grad_stage;
     }
     AdamArgs a{};
-    a.p = w.p; a.p_src = params_of(w); a.m = w.am; a.v = w.av; a.g = gdev; a.rep = w.rep;
+    a.p = w.p; a.p_src = params_of(w); a.m = w.am; a.v = w.av; a.rep = w.rep;
+    a.g = bf16 ? nullptr : static_cast<const float*>(gdev);
+    a.g16 = bf16 ? static_cast<const uint16_t*>(gdev) : nullptr;
     a.seg_end = c->seg_end; a.seg_decay = c->seg_decay; a.n_seg = c->n_seg;
     a.n = c->P;
     a.b1 = c->cfg.adam_b1; a.b2 = c->cfg.adam_b2;
@@ -404,6 +410,20 @@ int alsgd_inner_adamw(alsgd_ctx* c, uint32_t worker, const float* grads, int gra
     ALSGD_CUDA(c, launch_adamw(a, c->lc, c->stream));
     w.p_in_snapshot = false;
     return ALSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int alsgd_inner_adamw(alsgd_ctx* c, uint32_t worker, const float* grads, int grads_is_device,
+                      uint64_t step, float lr) {
+    return adamw_impl(c, worker, grads, false, grads_is_device, step, lr);
+}
+
+int alsgd_inner_adamw_bf16(alsgd_ctx* c, uint32_t worker, const uint16_t* grads, int grads_is_device,
+                           uint64_t step, float lr) {
+    return adamw_impl(c, worker, grads, true, grads_is_device, step, lr);
 }
 
 }  // extern "C"

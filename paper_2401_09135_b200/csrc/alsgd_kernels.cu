@@ -290,7 +290,13 @@ __device__ __forceinline__ SegCursor seg_find(uint64_t e, const AdamArgs& a) {
     return c;
 }
 
-template <int V>
+// bf16 -> fp32 is exact: the 16 bits are the upper half of the binary32 pattern.
+__device__ __forceinline__ float4 widen_bf16x4(uint2 b) {
+    return make_float4(__uint_as_float(b.x << 16), __uint_as_float(b.x & 0xFFFF0000u),
+                       __uint_as_float(b.y << 16), __uint_as_float(b.y & 0xFFFF0000u));
+}
+
+template <int V, bool G16>
 __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ AdamArgs a) {
     const uint64_t nvec = a.n >> 2;
     const uint64_t tile = (uint64_t)kBlock * V;
@@ -299,6 +305,7 @@ __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ A
     float4* __restrict__ m4 = reinterpret_cast<float4*>(a.m);
     float4* __restrict__ v4 = reinterpret_cast<float4*>(a.v);
     const float4* __restrict__ g4 = reinterpret_cast<const float4*>(a.g);
+    const uint2* __restrict__ g2 = reinterpret_cast<const uint2*>(a.g16);
     uint2* __restrict__ rep2 = reinterpret_cast<uint2*>(a.rep);
 
     SegCursor cur;
@@ -311,7 +318,7 @@ __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ A
         for (int k = 0; k < V; ++k) {
             const uint64_t i = t0 + (uint64_t)k * kBlock + threadIdx.x;
             if (i < nvec) {
-                g[k] = ld_stream(g4 + i);
+                g[k] = G16 ? widen_bf16x4(__ldcs(g2 + i)) : ld_stream(g4 + i);
                 p[k] = ld_stream(ps4 + i);
                 m[k] = ld_stream(m4 + i);
                 v[k] = ld_stream(v4 + i);
@@ -352,7 +359,8 @@ __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ A
         const uint64_t i = rem0 + threadIdx.x;
         SegCursor c = seg_find(i, a);
         float p = a.p_src[i], m = a.m[i], v = a.v[i];
-        adam_element(p, m, v, a.g[i], c.decay != 0, a);
+        const float gi = G16 ? __uint_as_float((uint32_t)a.g16[i] << 16) : a.g[i];
+        adam_element(p, m, v, gi, c.decay != 0, a);
         a.p[i] = p;
         a.m[i] = m;
         a.v[i] = v;
@@ -432,12 +440,12 @@ cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics
 cudaError_t launch_adamw(const AdamArgs& a, const LaunchCfg& lc, cudaStream_t s) {
     if (a.n == 0) return cudaSuccess;
     constexpr int V = 2;
-    auto kern = adamw_kernel<V>;
     unsigned grid = 1;
     cudaError_t e = grid_for(a.n, V, &grid);
     if (e != cudaSuccess) return e;
     (void)lc;
-    kern<<<grid, kBlock, 0, s>>>(a);
+    if (a.g16) adamw_kernel<V, true><<<grid, kBlock, 0, s>>>(a);
+    else adamw_kernel<V, false><<<grid, kBlock, 0, s>>>(a);
     return cudaGetLastError();
 }
 

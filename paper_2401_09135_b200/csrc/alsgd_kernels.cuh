@@ -49,7 +49,8 @@ struct AdamArgs {
     const float* p_src;        // parameters in (p itself, or the dispatch snapshot right after a dispatch)
     float* m;
     float* v;
-    const float* g;
+    const float* g;            // fp32 gradients, or null when g16 is used
+    const uint16_t* g16;       // bf16 gradients (bit patterns), or null
     uint16_t* rep;             // may be null
     const uint64_t* seg_end;   // device: ascending exclusive end of each weight-decay segment; last == n
     const uint32_t* seg_decay; // device: 1 if the segment is weight-decayed

@@ -346,6 +346,30 @@ def test_host_gradients_through_staging_equal_device_gradients():
     a.close(); b.close()
 
 
+@pytest.mark.parametrize("align", [1, 8])
+def test_bf16_gradients_equal_their_fp32_widening(align):
+    """bf16 gradients are widened exactly, so the step must equal the fp32 step on the widened values
+    (and therefore the oracle's), from device memory and through the host staging buffer."""
+    tensors = synth.ragged_tensors()
+    pair = Pair(tensors, 2, 4, 0.9, 0.7, align=align, grad_staging=True)
+    start(pair, SEED + 12)
+    for s in range(1, 4):
+        g = synth.zero_padding(synth.normal_vec(pair.P, 1e-2, SEED + 12, synth.STREAM_GRAD, sub=s), tensors, pair.offsets)
+        g16 = torch.from_numpy(g).to(torch.bfloat16)
+        wide = g16.to(torch.float32).numpy()
+        pair.ctx.alsgd_inner_adamw_bf16(0, g16.cuda(), s, 1e-3)
+        pair.orc.inner_adamw(0, pair.take(wide), s, 1e-3)
+        host = g16.pin_memory()
+        pair.ctx.alsgd_inner_adamw_bf16(1, host, s, 1e-3)
+        pair.ctx.alsgd_sync()
+        pair.orc.inner_adamw(1, pair.take(wide), s, 1e-3)
+        pair.check_worker(0, f"step {s} device bf16")
+        pair.check_worker(1, f"step {s} host bf16")
+    pair.arrive([0, 1], reseed=True)
+    pair.check_all("after arrival")
+    pair.close()
+
+
 def test_error_codes_leave_state_untouched():
     tensors = synth.flat_tensors(4096)
     ctx = B.Context(tensors, 3, 2, 0.9, 0.7)
