@@ -101,7 +101,8 @@ int alsgd_arena_bytes(const alsgd_tensor_desc* tensors, uint32_t n, uint32_t ali
 int alsgd_init(alsgd_ctx** out, const alsgd_tensor_desc* tensors, uint32_t n, uint32_t align_elems,
                const alsgd_config* cfg);
 
-/* Free the host bookkeeping.  Never touches the arena.  Does not wait for the stream. */
+/* Free the host bookkeeping (and, with ALSGD_CFG_GRAD_STAGING, the context's internal copy stream, after
+ * waiting for it).  Never touches the arena.  Does not wait for the caller's stream. */
 int alsgd_destroy(alsgd_ctx* ctx);
 
 /* Load theta^(0) (Algorithm 2: theta <- theta^(0)) / read theta.  P floats; is_device says where the
@@ -124,8 +125,10 @@ int alsgd_pull(alsgd_ctx* ctx, uint32_t worker);
  * flagged ALSGD_TENSOR_DECAY, bias correction from `step`, epsilon outside the root), followed by
  * the bf16 cast of the new parameters into the replica.
  *   grads            P fp32 values, 16-byte aligned, device or host (host needs
- *                    ALSGD_CFG_GRAD_STAGING; the copy is enqueued on the stream and the buffer is
- *                    borrowed until the stream reaches it)
+ *                    ALSGD_CFG_GRAD_STAGING; the vector is copied in pieces on an internal stream and the
+ *                    step on each piece is enqueued on the context's stream behind its copy, so copy and
+ *                    arithmetic overlap; the buffer is borrowed until the context's stream has passed
+ *                    this call; pinned memory keeps the call asynchronous)
  *   step             the worker's lifetime step count, >= 1
  *   lr               learning rate of this step
  * ALSGD_E_STATE if the worker was never dispatched, ALSGD_E_ARG if step = 0. */

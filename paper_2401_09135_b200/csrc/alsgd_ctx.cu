@@ -14,6 +14,7 @@ using namespace alsgd;
 namespace {
 
 constexpr uint64_t kSliceAlign = 256;  // bytes; every arena slice starts on this boundary
+constexpr int kStageChunks = 8;        // pieces a host gradient vector is copied in
 
 enum WorkerState : uint8_t { kNever = 0, kDispatched = 1, kArrived = 2 };
 
@@ -107,6 +108,11 @@ struct alsgd_ctx {
     float* mom = nullptr;
     float* delta = nullptr;
     float* grad_stage = nullptr;
+    // Host gradients are copied in chunks on a stream of their own so that the step on chunk i runs while
+    // chunk i+1 is still crossing PCIe.
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t stage_free = nullptr;               // main stream no longer reads the staging buffer
+    cudaEvent_t chunk_ready[kStageChunks] = {};
     std::vector<Worker> workers;
     // Dispatch snapshots: W slots of P floats.  Workers dispatched together (one grace window, one
     // theta) share one slot, so the snapshot is written once per window and read once per batch.
@@ -191,6 +197,13 @@ int copy_vec(alsgd_ctx* c, void* dst, const void* src, uint64_t bytes, bool host
 
 // Re-seed target: the worker's parameters and replica, plus (for one worker of the window) the
 // snapshot slot the whole window will share.
+void release_host_resources(alsgd_ctx* c) {
+    if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaStreamDestroy(c->copy_stream); c->copy_stream = nullptr; }
+    if (c->stage_free) { cudaEventDestroy(c->stage_free); c->stage_free = nullptr; }
+    for (int i = 0; i < kStageChunks; ++i)
+        if (c->chunk_ready[i]) { cudaEventDestroy(c->chunk_ready[i]); c->chunk_ready[i] = nullptr; }
+}
+
 void fill_seed(ArriveArgs& a, uint32_t slot, const Worker& w, float* snapshot, bool have_snapshots) {
     a.seed_p[slot] = have_snapshots ? nullptr : w.p;     // with snapshots the parameters are read from there
     a.seed_base[slot] = snapshot;
@@ -319,14 +332,23 @@ int alsgd_init(alsgd_ctx** out, const alsgd_tensor_desc* tensors, uint32_t n, ui
             if (e == cudaSuccess) e = cudaMemsetAsync(w.av, 0, sizeof(float) * P, c->stream);
             if (e == cudaSuccess && w.rep) e = cudaMemsetAsync(w.rep, 0, sizeof(uint16_t) * P, c->stream);
         }
+        if (e == cudaSuccess && c->grad_stage) {
+            e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->stage_free, cudaEventDisableTiming);
+            for (int i = 0; i < kStageChunks && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&c->chunk_ready[i], cudaEventDisableTiming);
+        }
         if (e != cudaSuccess) { c->last_cuda = (int)e; rc = ALSGD_E_CUDA; }
     }
-    if (rc != ALSGD_OK) { delete c; return rc; }
+    if (rc != ALSGD_OK) { release_host_resources(c); delete c; return rc; }
     *out = c;
     return ALSGD_OK;
 }
 
 int alsgd_destroy(alsgd_ctx* ctx) {
+    if (ctx) {
+        DeviceGuard g(ctx->cfg.device);
+        release_host_resources(ctx);
+    }
     delete ctx;
     return ALSGD_OK;
 }
@@ -389,25 +411,46 @@ int adamw_impl(alsgd_ctx* c, uint32_t worker, const void* grads, bool bf16, int 
     if (!grads_is_device && !c->grad_stage) return ALSGD_E_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(grads) % 16) return ALSGD_E_ARG;
     DeviceGuard g(c->cfg.device);
-    const void* gdev = grads;
-    if (!grads_is_device) {
-        const uint64_t bytes = (bf16 ? sizeof(uint16_t) : sizeof(float)) * c->P;
-        ALSGD_CUDA(c, cudaMemcpyAsync(c->grad_stage, grads, bytes, cudaMemcpyHostToDevice, c->stream));
-        gdev = c->grad_stage;
-    }
     AdamArgs a{};
-    a.p = w.p; a.p_src = params_of(w); a.m = w.am; a.v = w.av; a.rep = w.rep;
-    a.g = bf16 ? nullptr : static_cast<const float*>(gdev);
-    a.g16 = bf16 ? static_cast<const uint16_t*>(gdev) : nullptr;
+    a.rep = w.rep;
     a.seg_end = c->seg_end; a.seg_decay = c->seg_decay; a.n_seg = c->n_seg;
-    a.n = c->P;
     a.b1 = c->cfg.adam_b1; a.b2 = c->cfg.adam_b2;
     a.omb1 = 1.0f - a.b1; a.omb2 = 1.0f - a.b2;
     // Bias corrections: 1 - beta^step in double, rounded to fp32 once.
     a.bc1 = (float)(1.0 - std::pow((double)a.b1, (double)step));
     a.bc2 = (float)(1.0 - std::pow((double)a.b2, (double)step));
     a.eps = c->cfg.adam_eps; a.lr = lr; a.wd = c->cfg.adam_wd;
-    ALSGD_CUDA(c, launch_adamw(a, c->lc, c->stream));
+    const float* p_src = params_of(w);
+    const uint64_t esz = bf16 ? sizeof(uint16_t) : sizeof(float);
+    // One launch over [lo, lo + len) with the gradients at gsrc (device).
+    auto launch_range = [&](uint64_t lo, uint64_t len, const void* gsrc) -> cudaError_t {
+        a.p = w.p + lo; a.p_src = p_src + lo; a.m = w.am + lo; a.v = w.av + lo;
+        a.rep = w.rep ? w.rep + lo : nullptr;
+        a.g = bf16 ? nullptr : static_cast<const float*>(gsrc);
+        a.g16 = bf16 ? static_cast<const uint16_t*>(gsrc) : nullptr;
+        a.n = len;
+        a.seg_base = lo;
+        return launch_adamw(a, c->lc, c->stream);
+    };
+    if (grads_is_device) {
+        ALSGD_CUDA(c, launch_range(0, c->P, grads));
+    } else {
+        // Chunked: copy chunk i on the copy stream, run the step on it on the context's stream as soon as
+        // it has landed; the next chunk's copy overlaps that launch.
+        const uint64_t per = round_up((c->P + kStageChunks - 1) / kStageChunks, 1024);
+        ALSGD_CUDA(c, cudaEventRecord(c->stage_free, c->stream));          // earlier launches may still read the buffer
+        ALSGD_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->stage_free, 0));
+        uint8_t* stage = reinterpret_cast<uint8_t*>(c->grad_stage);
+        const uint8_t* src = static_cast<const uint8_t*>(grads);
+        int i = 0;
+        for (uint64_t lo = 0; lo < c->P; lo += per, ++i) {
+            const uint64_t len = (c->P - lo < per) ? c->P - lo : per;
+            ALSGD_CUDA(c, cudaMemcpyAsync(stage + lo * esz, src + lo * esz, len * esz, cudaMemcpyHostToDevice, c->copy_stream));
+            ALSGD_CUDA(c, cudaEventRecord(c->chunk_ready[i], c->copy_stream));
+            ALSGD_CUDA(c, cudaStreamWaitEvent(c->stream, c->chunk_ready[i], 0));
+            ALSGD_CUDA(c, launch_range(lo, len, stage + lo * esz));
+        }
+    }
     w.p_in_snapshot = false;
     return ALSGD_OK;
 }

@@ -328,7 +328,7 @@ __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ A
         for (int k = 0; k < V; ++k) {
             const uint64_t i = t0 + (uint64_t)k * kBlock + threadIdx.x;
             if (i >= nvec) continue;
-            const uint64_t e0 = i << 2;
+            const uint64_t e0 = a.seg_base + (i << 2);
             if (!have_cur) { cur = seg_find(e0, a); have_cur = true; }
             seg_seek(cur, e0, a);
             float* pf = reinterpret_cast<float*>(&p[k]);
@@ -357,7 +357,7 @@ __global__ void __launch_bounds__(kBlock) adamw_kernel(const __grid_constant__ A
     const uint64_t rem0 = nvec << 2;
     if (blockIdx.x == 0 && rem0 + threadIdx.x < a.n) {
         const uint64_t i = rem0 + threadIdx.x;
-        SegCursor c = seg_find(i, a);
+        SegCursor c = seg_find(a.seg_base + i, a);
         float p = a.p_src[i], m = a.m[i], v = a.v[i];
         const float gi = G16 ? __uint_as_float((uint32_t)a.g16[i] << 16) : a.g[i];
         adam_element(p, m, v, gi, c.decay != 0, a);

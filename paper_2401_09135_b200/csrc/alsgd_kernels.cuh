@@ -55,7 +55,8 @@ struct AdamArgs {
     const uint64_t* seg_end;   // device: ascending exclusive end of each weight-decay segment; last == n
     const uint32_t* seg_decay; // device: 1 if the segment is weight-decayed
     uint32_t n_seg;
-    uint64_t n;
+    uint64_t n;                // elements in this launch
+    uint64_t seg_base;         // flat index of this launch's first element (segment ends are flat indices)
     float b1, b2, omb1, omb2, bc1, bc2, eps, lr, wd;
 };
 
