@@ -370,6 +370,50 @@ def test_bf16_gradients_equal_their_fp32_widening(align):
     pair.close()
 
 
+def test_nothing_is_written_past_the_end_of_a_slice():
+    """Every arena slice starts on a 256-byte boundary; with P = 4099 + ... odd sizes the bytes between the end
+    of a slice and the next boundary belong to nobody.  They are filled with a canary before the run and must
+    still hold it afterwards (vector stores, tails, re-seed and bf16 stores all end exactly at P)."""
+    tensors = synth.ragged_tensors()
+    W = 5
+    pair = Pair(tensors, W, 2, 0.9, 0.7, align=1)
+    P = pair.P
+    assert P % 64 != 0
+    ctx = pair.ctx
+    arena, base = ctx.arena, ctx.arena.data_ptr()
+    gaps = []
+
+    def gap_after(tensor):
+        if tensor is None:
+            return
+        end = tensor.data_ptr() + tensor.numel() * tensor.element_size() - base
+        stop = (end + 255) // 256 * 256
+        if stop > end and stop <= arena.numel():
+            gaps.append((end, stop))
+
+    for v in ctx.alsgd_state_ptrs():
+        gap_after(v)
+    for w in range(W):
+        for v in ctx.alsgd_worker_state_ptrs(w).values():
+            gap_after(v)
+    assert len(gaps) >= 3 + 5 * W - W
+    ctx.alsgd_sync()
+    for lo, hi in gaps:
+        arena[lo:hi] = 0xA5
+    start(pair, SEED + 13)
+    life = [0] * W
+    for b, ids in enumerate([[0, 1], [2], [3, 4, 0], [1, 2, 3, 4, 0], [2, 4]]):
+        for w in ids:
+            life[w] += 1
+            g = synth.zero_padding(synth.normal_vec(P, 1e-2, SEED + 13, synth.STREAM_GRAD, sub=w * 10 + life[w]), tensors, pair.offsets)
+            pair.inner_adamw(w, dev(g), g, life[w], 1e-3)
+        pair.arrive(ids, reseed=True, norm=True)
+    pair.check_all("canary run")
+    for lo, hi in gaps:
+        assert bool((arena[lo:hi] == 0xA5).all()), f"bytes {lo}..{hi} of the arena were overwritten"
+    pair.close()
+
+
 def test_error_codes_leave_state_untouched():
     tensors = synth.flat_tensors(4096)
     ctx = B.Context(tensors, 3, 2, 0.9, 0.7)
