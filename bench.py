@@ -411,6 +411,60 @@ def main_ksweep(args):
                       "peak_gbs": peak, "peak_source": f"of {which}", "unit": "GB/s", "rounds_timed": len(ev), "sweep": out}), flush=True)
 
 
+def main_layouts(args):
+    """Per-kernel throughput on layouts shaped like the paper's 20M-150M decoder transformers (2 workers, N = 4):
+    20 AdamW steps and 20 single arrivals with fused re-seed each, CUDA events, after 4 warm-up launches.
+    Below ~30M elements one fp32 buffer fits in L2, so those rows are not HBM-roofline figures."""
+    import torch
+    from paper_2401_09135_b200 import binding as B, synth
+    torch.cuda.set_device(0)
+    peak, which = measured_peak()
+    out = []
+    for name, tensors in (("23M (6L, d384, ff1536)", synth.layout_23m()), ("paper 60M (3L, h896, 16x64)", synth.layout_paper_60m()),
+                          ("110M (12L, d768, ff3072)", synth.layout_110m()), ("paper 150M (12L, h896, 16x64)", synth.layout_paper_150m())):
+        ctx = B.Context(tensors, 2, 4, 0.9, 0.7)
+        P = ctx.P
+        ctx.alsgd_set_global(synth.theta0(tensors, ctx.offsets, P))
+        g = [torch.from_numpy(synth.normal_vec(P, 1e-2, synth.SEED, synth.STREAM_GRAD, sub=i)).cuda() for i in range(2)]
+        for w in range(2):
+            ctx.alsgd_pull(w)
+        step = 0
+
+        def adam(n):
+            nonlocal step
+            for i in range(n):
+                step += 1
+                ctx.alsgd_inner_adamw(i % 2, g[i % 2], step, 1e-3)
+
+        res = {"layout": name, "P": P}
+        adam(4)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); adam(20); e1.record(); torch.cuda.synchronize()
+        times = {"adamw": e0.elapsed_time(e1) / 20}
+        # arrivals: one AdamW step of the arriving worker (untimed) before each, so that the arrival reads the
+        # worker's own parameters and not the snapshot it was dispatched with
+        pairs = []
+        for i in range(24):
+            w = i % 2
+            step += 1
+            ctx.alsgd_inner_adamw(w, g[w], step, 1e-3)
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            ctx.alsgd_arrive([w], B.ARRIVE_RESEED, want_info=False)
+            a1.record()
+            pairs.append((a0, a1))
+        torch.cuda.synchronize()
+        times["arrive_reseed"] = sum(x.elapsed_time(y) for x, y in pairs[4:]) / 20
+        for key, bpp in (("adamw", ADAMW_BYTES), ("arrive_reseed", 30.0)):
+            ms = times[key]
+            res[key] = {"ms": ms, "params_per_s": P / (ms * 1e-3), "gbs": bpp * P / (ms * 1e-3) / 1e9,
+                        "frac_of_measured": bpp * P / (ms * 1e-3) / 1e9 / peak, "frac_of_8TBs": bpp * P / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS}
+        out.append(res)
+        ctx.close(); del ctx, g
+        torch.cuda.empty_cache()
+    print(json.dumps({"peak_gbs": peak, "peak_source": f"of {which}", "layouts": out}), flush=True)
+
+
 def main_cpu_kernels(args):
     """The oracle's two loops timed per kernel on the host: one core as written, and the same scalar
     loops range-split over all host cores (exact, the path is elementwise)."""
@@ -462,12 +516,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ksweep", action="store_true", help="arrival-batch sweep (k = 1, 2, 4, 8) with 8 resident workers")
+    ap.add_argument("--layouts", action="store_true", help="per-kernel throughput on 23M / 60M / 110M / 150M layouts")
     ap.add_argument("--cpu-kernels", action="store_true", help="time the oracle's loops per kernel on the host cores")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.cpu_kernels:
+    if args.layouts:
+        main_layouts(args)
+    elif args.cpu_kernels:
         main_cpu_kernels(args)
     elif args.ksweep:
         main_ksweep(args)

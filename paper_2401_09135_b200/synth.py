@@ -59,6 +59,37 @@ def transformer_tensors(vocab: int, d_model: int, d_ff: int, n_layers: int):
     return t
 
 
+def paper_tensors(vocab: int, hidden: int, n_heads: int, kv_size: int, n_layers: int, ff_mult: int = 4):
+    """Tensor list with the numbers of the paper's Table 6 (layers, hidden dim, heads, K/V size, vocab):
+    attention width n_heads * kv_size (which differs from the hidden dim for the 60M / 150M models),
+    feed-forward width ff_mult * hidden, tied embedding, LayerNorm gain+bias, no linear biases."""
+    d_attn = n_heads * kv_size
+    t = [Tensor("tok_emb", vocab * hidden, True, "matrix")]
+    for l in range(n_layers):
+        t.append(Tensor(f"l{l}.ln1.g", hidden, False, "gain"))
+        t.append(Tensor(f"l{l}.ln1.b", hidden, False, "bias"))
+        for w in ("wq", "wk", "wv"):
+            t.append(Tensor(f"l{l}.{w}", hidden * d_attn, True, "matrix"))
+        t.append(Tensor(f"l{l}.wo", d_attn * hidden, True, "matrix"))
+        t.append(Tensor(f"l{l}.ln2.g", hidden, False, "gain"))
+        t.append(Tensor(f"l{l}.ln2.b", hidden, False, "bias"))
+        t.append(Tensor(f"l{l}.w_ff1", hidden * ff_mult * hidden, True, "matrix"))
+        t.append(Tensor(f"l{l}.w_ff2", ff_mult * hidden * hidden, True, "matrix"))
+    t.append(Tensor("lnf.g", hidden, False, "gain"))
+    t.append(Tensor("lnf.b", hidden, False, "bias"))
+    return t
+
+
+def layout_paper_60m():
+    """Table 6, 60M column: 3 layers, hidden 896, 16 heads of size 64, vocab 32000 (~59M elements)."""
+    return paper_tensors(32000, 896, 16, 64, 3)
+
+
+def layout_paper_150m():
+    """Table 6, 150M column: 12 layers, hidden 896, 16 heads of size 64, vocab 32000 (~150M elements)."""
+    return paper_tensors(32000, 896, 16, 64, 12)
+
+
 def layout_23m():
     """~23M-parameter layout: 6 layers, d_model 384, d_ff 1536, vocab 32000 (22 914 816 elements)."""
     return transformer_tensors(32000, 384, 1536, 6)
