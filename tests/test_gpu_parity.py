@@ -370,6 +370,39 @@ def test_bf16_gradients_equal_their_fp32_widening(align):
     pair.close()
 
 
+def test_extreme_values_denormals_signed_zeros_overflow():
+    """The bit-for-bit claim at the edges of binary32: denormals (no flush to zero on either side), signed
+    zeros, values whose products overflow to infinity or underflow to zero, and huge/tiny mixes in AdamW's
+    divisions and square root."""
+    P = 8192
+    tensors = [synth.Tensor("a", P // 2, True, "matrix"), synth.Tensor("b", P // 2, False, "gain")]
+    pair = Pair(tensors, 3, 2, 0.9, 0.7, c=0.25, align=1)
+    specials = np.array([0.0, -0.0, 1e-45, -1e-45, 1e-40, -3e-39, 1.1754944e-38, -1.1754942e-38, 1e-30, -1e-20,
+                         1e-10, 1.0, -1.0, 3.0, 1e10, -1e19, 1e20, -1e30, 3e38, -3.4028235e38, 65504.0, 1e-7], np.float32)
+    r = np.random.default_rng(21)
+
+    def special_vec():
+        return np.ascontiguousarray(specials[r.integers(0, specials.shape[0], P)])
+
+    with np.errstate(all="ignore"):
+        pair.set_global(special_vec())
+        for w in range(3):
+            pair.pull(w)
+        for rnd in range(4):
+            for w in range(3):
+                z = special_vec()
+                pair.perturb(w, dev(z), z)
+                g = special_vec()
+                pair.inner_adamw(w, dev(g), g, rnd + 1, 1e-3)
+            pair.arrive([[0, 1, 2], [2, 0], [1], [1, 2, 0]][rnd], reseed=True, norm=True)
+            pair.check_all(f"round {rnd}")
+    th = pair.orc.theta
+    assert np.isinf(th).any() or np.isnan(th).any()          # the inputs did reach overflow
+    v = pair.orc.av[0]
+    assert ((v > 0) & (v < 1.1754944e-38)).any()             # ... and the denormal range (second moments of tiny gradients)
+    pair.close()
+
+
 def test_nothing_is_written_past_the_end_of_a_slice():
     """Every arena slice starts on a 256-byte boundary; with P = 4099 + ... odd sizes the bytes between the end
     of a slice and the next boundary belong to nobody.  They are filled with a canary before the run and must
