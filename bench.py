@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter from the committed ncu captures
 # (profiles/), valid only for the kernel source they were taken from.
 NCU_TRAFFIC = {
-    "src_sha256": "64d60c0cadb2407f2d55c5915c0a2b18502224063a9633a32f0c771181288bc0",
+    "src_sha256": "096949379a0ffd9f559f91c7bc7f061aede597ccb5d156faabf1363cc667106a",
     "adamw_bytes_per_param": 28.90,     # ncu capture at P = 50.3M elements, scaled by P
     "arrive_bytes_per_param": 28.90,    # same capture, K = 1, average over one Delayed-Nesterov cycle
 }

@@ -11,7 +11,8 @@
 //
 // Arithmetic contract: every fp32 operation is a separate IEEE-754 round-to-nearest operation in
 // the order Algorithm 3 states it (this file is compiled with -fmad=false, IEEE division and
-// square root, no flush-to-zero), so results do not depend on the launch shape.
+// square root, no flush-to-zero), so results do not depend on the launch shape.  The only fused
+// multiply-adds are the explicit ones of the optional diagnostics, which feed no state.
 #include "alsgd_kernels.cuh"
 
 #include <cuda_runtime.h>
@@ -189,8 +190,8 @@ __global__ void __launch_bounds__(kBlock) arrive_kernel(const __grid_constant__ 
     }
 
     // ---- optional diagnostics: one partial sum per block per arrival, added up in a fixed order by
-    //      the two diag_reduce kernels (no atomics: 10^5 blocks adding into a handful of addresses serialise in
-    //      one L2 slice and cost up to 40 % of the pass); one flag per arrival
+    //      the two diag_reduce kernels (no floating-point atomics, so the norm is reproducible run to
+    //      run); one flag per arrival, raised by an atomicOr only when an entry is Inf or NaN
     if (DIAG && K > 0) {
         __shared__ float warp_sum[kBlock / 32][KK];
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
