@@ -15,10 +15,35 @@ from . import binding as B
 from . import synth
 
 
+def batches_case():
+    n = 32 * 1024 * 1024
+    tensors = synth.flat_tensors(n)
+    W = 8
+    ctx = B.Context(tensors, W, 8, 0.9, 0.7)
+    ctx.alsgd_set_global(synth.theta0(tensors, ctx.offsets, ctx.P))
+    g = torch.from_numpy(synth.normal_vec(ctx.P, 1e-2, synth.SEED, synth.STREAM_GRAD)).cuda()
+    for w in range(W):
+        ctx.alsgd_pull(w)
+    for w in range(W):
+        ctx.alsgd_inner_adamw(w, g, 1, 1e-3)
+    ctx.alsgd_arrive([0, 1, 2, 3], B.ARRIVE_RESEED, want_info=False)     # first of the cycle, four distinct snapshots
+    ctx.alsgd_arrive([4, 5, 6, 7], B.ARRIVE_RESEED, want_info=False)     # ends the cycle of N = 8 (boundary inside)
+    for w in range(W):
+        ctx.alsgd_inner_adamw(w, g, 2, 1e-3)
+    ctx.alsgd_arrive(list(range(W)), B.ARRIVE_RESEED, want_info=False)   # whole cycle in one pass, two shared snapshots
+    ctx.alsgd_sync()
+    print(f"batches case done: P={ctx.P}, t={ctx.alsgd_counters()[0]}")
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--elems", type=int, default=48 * 1024 * 1024)
+    ap.add_argument("--batches", action="store_true",
+                    help="8 workers on 32Mi elements (4.3 GB): one AdamW step each, two batches of 4, one AdamW step each, one batch of 8")
     args = ap.parse_args()
+    if args.batches:
+        return batches_case()
     n = args.elems
     tensors = [synth.Tensor("w0", n // 2, True, "matrix"), synth.Tensor("g0", 4096, False, "gain"),
                synth.Tensor("w1", n - n // 2 - 4096, True, "matrix")]
