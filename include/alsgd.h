@@ -213,9 +213,12 @@ typedef struct alsgd_worker_ptrs {
 } alsgd_worker_ptrs;
 
 /* Borrowed device pointers into the arena, valid until alsgd_destroy, for a harness that perturbs
- * workers and reads results.  Right after a momentum boundary Delta is zero by definition and the
- * library may not have written those zeros yet; this call enqueues that fill first, so every read
- * ordered after it on the context's stream sees Algorithm 3's Delta. */
+ * workers and reads results.  Two stores are deferred by the library and made good here before a
+ * pointer is handed out, so every access ordered after the call on the context's stream sees the
+ * defined state: right after a momentum boundary Delta is zero by definition but those zeros may
+ * not have been written yet (alsgd_state_ptrs enqueues the fill); right after a dispatch a worker's
+ * parameters equal its snapshot and may not have been copied into `p` yet
+ * (alsgd_worker_state_ptrs enqueues the copy). */
 int alsgd_state_ptrs(alsgd_ctx* ctx, alsgd_ptrs* out);
 int alsgd_worker_state_ptrs(alsgd_ctx* ctx, uint32_t worker, alsgd_worker_ptrs* out);
 
