@@ -101,9 +101,15 @@ def cast_bf16(src: np.ndarray) -> np.ndarray:
     return out
 
 
+OUTER_DN, OUTER_BUFFERED, OUTER_SGDM = 0, 1, 2
+
+
 def dn_arrive(theta, m, Delta, base, p, t, N, beta, eps, c=0.0, pg_current=False, weight=1.0,
               dc_lambda=0.0, buffered=False, lo=0, hi=None) -> bool:
-    """One arrival of Algorithm 3 in place on float32 arrays; returns the boundary flag."""
+    """One arrival of Algorithm 3 in place on float32 arrays; returns the boundary flag.
+
+    buffered: False / OUTER_DN = Delayed Nesterov; True / OUTER_BUFFERED = "Async. Buffer" (Nesterov step
+    on the buffer mean at every N-th arrival); OUTER_SGDM = the same with the SGD Momentum step."""
     hi = theta.shape[0] if hi is None else hi
     for a in (theta, m, Delta, p):
         assert a.dtype == np.float32
@@ -113,7 +119,7 @@ def dn_arrive(theta, m, Delta, base, p, t, N, beta, eps, c=0.0, pg_current=False
     return bool(lib().orc_dn_arrive(_p(theta, _f32p), _p(m, _f32p), _p(Delta, _f32p), _p(base, _f32p),
                                     _p(p, _f32p), lo, hi, int(t), int(N), float(beta), float(eps),
                                     float(c), int(bool(pg_current)), float(weight), float(dc_lambda),
-                                    int(bool(buffered))))
+                                    int(buffered)))
 
 
 def pg_norm2(theta, base, p, pg_current=False, lo=0, hi=None):

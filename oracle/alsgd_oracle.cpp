@@ -20,7 +20,8 @@
 //   orc_shard_probs Eq. 2 hand values, normalisation, start-up and balanced special cases.
 //   orc_poly_weight, weight / dc_lambda / buffered arguments of orc_dn_arrive: formulas of Section 4
 //                   ("Existing Fixes"): hand cases, zero-drift and homogeneity properties, buffered
-//                   N = 1 == Eq. 4, buffered == Delayed Nesterov at cycle ends.
+//                   N = 1 == Eq. 4, buffered == Delayed Nesterov at cycle ends; SGD Momentum outer step:
+//                   hand trace, theta' = theta - eps m', beta = 0 == plain SGD, geometric closed form.
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -79,6 +80,10 @@ float orc_between_weight(float beta, float c) {                   // c * beta
 //   dc_lambda   delay-compensation strength (Section 4, fix 3); 0 disables it.
 //   buffered    1: "Async. Buffer" (Section 4, fix 4): theta moves only at the boundary, by one
 //               Nesterov step (Eq. 4) on the buffer mean.
+//               2: the same buffered structure with the "SGD Momentum" outer step of Section 4's
+//               optimizer grid, which the text under Eq. 4 defines by its difference from Nesterov:
+//               momentum weight beta instead of beta^2, gradient weight 1 instead of 1 + beta, i.e.
+//               m' = beta m + g, theta' = theta - eps (beta m + g).  N = 1 applies it at every arrival.
 // Returns 1 when this arrival is a momentum boundary ((t+1) % N == 0), else 0.
 // ---------------------------------------------------------------------------------------------
 int orc_dn_arrive(float* theta, float* m, float* Delta, const float* base, const float* p,
@@ -102,7 +107,12 @@ int orc_dn_arrive(float* theta, float* m, float* Delta, const float* base, const
             if (boundary) {
                 const float mean = d * invN;
                 const float mn = (beta * m[i]) + mean;            // Eq. 4, momentum
-                const float u = ((beta * beta) * m[i]) + ((1.0f + beta) * mean);
+                float u;
+                if (buffered == 2) {
+                    u = (beta * m[i]) + mean;                     // SGD Momentum: weights beta and 1
+                } else {
+                    u = ((beta * beta) * m[i]) + ((1.0f + beta) * mean);   // Nesterov: beta^2 and 1 + beta
+                }
                 theta[i] = theta[i] - (eps * u);
                 m[i] = mn;
                 Delta[i] = 0.0f;

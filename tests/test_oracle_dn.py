@@ -268,3 +268,28 @@ def test_pg_norm_and_nonfinite_flag():
     p[1] = np.inf
     s, bad = oracle.pg_norm2(theta, base, p)
     assert bad == 1
+
+
+def test_pg_norm_in_current_mode_is_taken_against_the_running_theta():
+    # the norm of theta - p, whatever the dispatch snapshot holds: (1 - 0.5)^2 + (2 - 2.5)^2 = 0.5
+    theta = np.array([1.0, 2.0], np.float32)
+    base = np.array([99.0, -99.0], np.float32)
+    p = np.array([0.5, 2.5], np.float32)
+    s, bad = oracle.pg_norm2(theta, base, p, pg_current=True)
+    assert s == 0.5 and bad == 0
+    s, bad = oracle.pg_norm2(theta, base, p, pg_current=False)
+    assert s == 98.5 ** 2 + 101.5 ** 2 and bad == 0
+    # inside a batch the second arrival's pseudo-gradient is against theta after the first:
+    # N=4 beta=0.5 eps=0.5, theta=1, workers at 0.5 and 0.75.  First: g = 0.5, theta = 1 - 0.5*0.5/4 = 0.9375.
+    # Second: g = 0.9375 - 0.75 = 0.1875 (against the dispatch model it would be 0.25).
+    srv = oracle.OracleServer(3, 2, 4, 0.5, 0.5, pg_current=True)
+    srv.set_global(np.ones(3, np.float32))
+    srv.pull(0); srv.pull(1)
+    srv.p[0][:] = 0.5
+    srv.p[1][:] = 0.75
+    info = srv.arrive([0, 1], norm=True)
+    assert info[0]["gnorm2"] == 3 * 0.25 and info[1]["gnorm2"] == 3 * 0.1875 ** 2
+    np.testing.assert_array_equal(srv.Delta, np.float32(0.6875))
+    srv.p[0][1] = np.nan                                   # re-dispatched at theta; one poisoned entry
+    info = srv.arrive([0], norm=True)
+    assert info[0]["nonfinite"] == 1

@@ -22,7 +22,8 @@ DN_PINS = [dn.test_hand_trace_c0_eight_elements, dn.test_hand_trace_c_quarter_ei
            dn.test_momentum_weights_sum_to_beta_over_a_cycle,
            lambda: dn.test_matches_exact_unrolled_sums(3, 0.25), lambda: dn.test_matches_exact_unrolled_sums(4, 0.0),
            dn.test_one_cycle_equals_synchronous_diloco_with_nesterov, dn.test_current_mode_uses_running_theta,
-           dn.test_server_bookkeeping_ticks_boundaries_staleness, dn.test_pg_norm_and_nonfinite_flag]
+           dn.test_server_bookkeeping_ticks_boundaries_staleness, dn.test_pg_norm_and_nonfinite_flag,
+           dn.test_pg_norm_in_current_mode_is_taken_against_the_running_theta]
 ADAM_PINS = [misc.test_adamw_hand_case, misc.test_adamw_first_step_is_sign_step_without_eps_and_decay,
              misc.test_adamw_constant_gradient_keeps_sign_stepping, misc.test_adamw_zero_gradient_is_pure_decoupled_decay,
              misc.test_adamw_against_library_adamw_in_double]
@@ -33,7 +34,8 @@ HOST_PINS = [misc.test_shard_sampling_eq2, misc.test_dylu_values, misc.test_lr_s
              misc.test_schedule_stops_at_t_max_local_updates]
 VAR_PINS = [var.test_buffered_hand_trace, var.test_buffered_with_N1_is_plain_nesterov_and_matches_dn_at_cycle_ends,
             var.test_delay_compensation_hand_case_and_zero_drift, var.test_weighted_arrival_hand_case_and_homogeneity,
-            var.test_poly_weights_and_threshold_bookkeeping]
+            var.test_poly_weights_and_threshold_bookkeeping, var.test_delay_compensation_comes_before_the_staleness_weight,
+            var.test_sgd_momentum_outer_step_hand_trace, var.test_sgd_momentum_outer_step_properties]
 
 # (name, text to find, replacement, which occurrence (None = all), pins that must catch it)
 MUTANTS = [
@@ -78,6 +80,16 @@ MUTANTS = [
     ("buffered step with beta, not beta^2", "((beta * beta) * m[i])", "(beta * m[i])", None, VAR_PINS),
     ("buffered theta moves between boundaries", "} else {\n                Delta[i] = d;\n            }\n            continue;", "} else {\n                theta[i] = theta[i] - (eps * gn);\n                Delta[i] = d;\n            }\n            continue;", None, VAR_PINS),
     ("weight ignored", "if (weight != 1.0f) g = weight * g;", "", None, VAR_PINS),
+    ("current mode ignored in the norm", "const float start = pg_current ? theta[i] : base[i];\n        const float g", "const float start = base[i];\n        const float g", None, DN_PINS),
+    ("norm of the sum, not sum of squares", "acc += (double)g * (double)g;", "acc += (double)g;", None, DN_PINS),
+    ("non-finite test misses infinities", "if (!std::isfinite(g)) bad = 1;", "if (std::isnan(g)) bad = 1;", None, DN_PINS),
+    ("SGD momentum step with beta^2", "u = (beta * m[i]) + mean;", "u = ((beta * beta) * m[i]) + mean;", None, VAR_PINS),
+    ("SGD momentum step with gradient weight 1 + beta", "u = (beta * m[i]) + mean;", "u = (beta * m[i]) + ((1.0f + beta) * mean);", None, VAR_PINS),
+    ("SGD momentum mode falls through to Nesterov", "if (buffered == 2) {", "if (buffered == 3) {", None, VAR_PINS),
+    ("weight applied before delay compensation",
+     "            g = g + ((dc_lambda * (g * g)) * drift);\n        }\n        if (weight != 1.0f) g = weight * g;",
+     "            const float gw = weight * g;\n            g = gw + ((dc_lambda * (gw * gw)) * drift);\n        } else if (weight != 1.0f) g = weight * g;",
+     None, VAR_PINS),
 ]
 
 
