@@ -465,6 +465,29 @@ def main_layouts(args):
     print(json.dumps({"peak_gbs": peak, "peak_source": f"of {which}", "layouts": out}), flush=True)
 
 
+def main_shape_sweep(args):
+    """Times many launch shapes of the product's kernel bodies (libalsgd_sweep.so) at the 110M size: threads per
+    block, vectors per thread, resident-block caps, one tile per block against a persistent loop, scalar against
+    packed two-lane arithmetic, per-arrival against shared dispatch snapshot, with and without diagnostics.
+    Prints one JSON object: every row, and the best shape per (kernel, K, snapshot mode, diagnostics)."""
+    import torch
+    from paper_2401_09135_b200 import sweep
+    torch.cuda.set_device(0)
+    n = args.sweep_elems
+    peak, which = measured_peak()
+    rows = sweep.run(n, reps=args.sweep_reps, warmup=3,
+                     log=(lambda r: print(json.dumps(r), file=sys.stderr, flush=True)) if args.verbose else None)
+    best = {}
+    for r in rows:
+        if r["persistent"]:
+            continue
+        key = ("adamw" if r["kind"] == sweep.KIND_ADAMW else f"arrive K={r['K']} base={sweep.BASE_NAMES[r['base_mode']]}") + (" diag" if r["diag"] else "")
+        if key not in best or r["gbs"] > best[key]["gbs"]:
+            best[key] = r
+    print(json.dumps({"elements": n, "reps": args.sweep_reps, "peak_gbs": peak, "peak_source": f"of {which}",
+                      "unit": "GB/s on algorithmic bytes", "best": best, "rows": rows}), flush=True)
+
+
 def main_cpu_kernels(args):
     """The oracle's two loops timed per kernel on the host: one core as written, and the same scalar
     loops range-split over all host cores (exact, the path is elementwise)."""
@@ -518,11 +541,17 @@ def main():
     ap.add_argument("--ksweep", action="store_true", help="arrival-batch sweep (k = 1, 2, 4, 8) with 8 resident workers")
     ap.add_argument("--layouts", action="store_true", help="per-kernel throughput on 23M / 60M / 110M / 150M layouts")
     ap.add_argument("--cpu-kernels", action="store_true", help="time the oracle's loops per kernel on the host cores")
+    ap.add_argument("--shape-sweep", action="store_true", help="time the launch shapes of libalsgd_sweep.so")
+    ap.add_argument("--sweep-elems", type=int, default=109_549_056)
+    ap.add_argument("--sweep-reps", type=int, default=10)
+    ap.add_argument("--verbose", action="store_true")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.layouts:
+    if args.shape_sweep:
+        main_shape_sweep(args)
+    elif args.layouts:
         main_layouts(args)
     elif args.cpu_kernels:
         main_cpu_kernels(args)

@@ -9,7 +9,12 @@
  *
  * Conventions
  *   - Every function returns ALSGD_OK (0) or a negative alsgd_status.  Nothing throws, aborts,
- *     traps or prints.  On an error the context is left as it was before the call.
+ *     traps or prints.  Arguments are checked before anything is enqueued, so ALSGD_E_ARG, _RANGE,
+ *     _STATE, _NOMEM and _UNSUPPORTED leave the context exactly as it was.  ALSGD_E_CUDA from a call
+ *     whose first launch failed does too; if a later launch of the same call fails (an arrival batch
+ *     larger than one pass, a host gradient copied in pieces) the device state is already ahead of
+ *     the host bookkeeping: the context then refuses every further state-changing call with
+ *     ALSGD_E_STATE and can only be read, destroyed or re-filled by alsgd_import_state.
  *   - "host" / "device" is stated for every pointer.  The arena and the stream belong to the
  *     caller; the context owns only host bookkeeping.  No entry point allocates device memory
  *     (alsgd_init and alsgd_destroy allocate and free host memory only).
@@ -34,7 +39,8 @@ typedef enum alsgd_status {
     ALSGD_E_STATE = -3,  /* call not allowed in the current state (e.g. arrival of a worker never dispatched) */
     ALSGD_E_CUDA = -4,   /* a CUDA runtime call failed; see alsgd_last_cuda_error */
     ALSGD_E_NOMEM = -5,  /* arena too small, or host allocation failed */
-    ALSGD_E_UNSUPPORTED = -6
+    ALSGD_E_UNSUPPORTED = -6,
+    ALSGD_E_BOUNDS = -7  /* debug build only: a kernel access fell outside the arena and was skipped (alsgd_sync) */
 } alsgd_status;
 
 /* Text for a status code (static storage, host). */
@@ -74,6 +80,16 @@ typedef struct alsgd_ctx alsgd_ctx;
 #define ALSGD_CFG_GRAD_STAGING 2u  /* reserve a P-element fp32 staging buffer so that alsgd_inner_adamw accepts host gradients */
 #define ALSGD_CFG_OUTER_BUFFERED 4u /* "Async. Buffer" of Section 4 instead of Delayed Nesterov: Delta accumulates every arrival,
                                        theta and m move only on every N-th, by the Nesterov step of Eq. 4 on Delta/N; c is unused */
+#define ALSGD_CFG_OUTER_SGDM 8u     /* "SGD Momentum" of Section 4's outer-optimizer grid, in the same buffered structure: on every
+                                       N-th arrival m <- beta m + g, theta <- theta - eps (beta m + g) with g = Delta/N, i.e. Eq. 4
+                                       with beta in place of beta^2 and 1 in place of 1 + beta (the text under Eq. 4).  N = 1 applies
+                                       it at every arrival, as the paper's grid did; beta = 0 is plain outer SGD.  c is unused.
+                                       Not together with ALSGD_CFG_OUTER_BUFFERED. */
+#define ALSGD_CFG_STABLE_PTRS 16u   /* no deferred stores: every worker keeps a snapshot of its own and its parameters are written
+                                       at every dispatch, Delta's zeros are written at every boundary, so the pointers of
+                                       alsgd_state_ptrs / alsgd_worker_state_ptrs stay valid and current for the context's lifetime.
+                                       Costs 4 (parameters) + 4 (own snapshot) bytes per parameter per dispatched worker instead of
+                                       4 per window, and 4 per boundary. */
 
 typedef struct alsgd_config {
     uint32_t n_workers;  /* W >= 1 replicas resident in the arena */
@@ -102,7 +118,9 @@ int alsgd_init(alsgd_ctx** out, const alsgd_tensor_desc* tensors, uint32_t n, ui
                const alsgd_config* cfg);
 
 /* Free the host bookkeeping (and, with ALSGD_CFG_GRAD_STAGING, the context's internal copy stream, after
- * waiting for it).  Never touches the arena.  Does not wait for the caller's stream. */
+ * waiting for it).  Never touches the arena.  Does not wait for the caller's stream: kernels of earlier
+ * calls may still be running on it, so the caller synchronises that stream (or calls alsgd_sync first)
+ * before it frees or reuses the arena. */
 int alsgd_destroy(alsgd_ctx* ctx);
 
 /* Load theta^(0) (Algorithm 2: theta <- theta^(0)) / read theta.  P floats; is_device says where the
@@ -212,13 +230,23 @@ typedef struct alsgd_worker_ptrs {
     uint16_t* replica; /* device, P bf16 bit patterns (NULL without ALSGD_CFG_REPLICA_BF16) */
 } alsgd_worker_ptrs;
 
-/* Borrowed device pointers into the arena, valid until alsgd_destroy, for a harness that perturbs
- * workers and reads results.  Two stores are deferred by the library and made good here before a
- * pointer is handed out, so every access ordered after the call on the context's stream sees the
- * defined state: right after a momentum boundary Delta is zero by definition but those zeros may
- * not have been written yet (alsgd_state_ptrs enqueues the fill); right after a dispatch a worker's
- * parameters equal its snapshot and may not have been copied into `p` yet
- * (alsgd_worker_state_ptrs enqueues the copy). */
+/* Borrowed device pointers into the arena, for a harness that perturbs workers and reads results.
+ * theta, m, adam_m, adam_v and replica always hold the current state and stay valid until
+ * alsgd_destroy.  `delta`, `p` and `base` are different: the library defers two stores and shares
+ * snapshots, and makes the state good only at the moment of this call.
+ *   - Right after a momentum boundary Delta is zero by definition but the zeros may not have been
+ *     written; alsgd_state_ptrs enqueues the fill.  `delta` read after a LATER boundary without a new
+ *     alsgd_state_ptrs call may show the pre-boundary buffer.
+ *   - Right after a dispatch (alsgd_pull, alsgd_arrive with RESEED) a worker's parameters equal its
+ *     snapshot and are not copied into `p`; alsgd_worker_state_ptrs enqueues that copy (P floats).
+ *     A `p` pointer kept across a LATER dispatch of that worker shows the previous round's
+ *     parameters until the next alsgd_worker_state_ptrs, alsgd_set_worker_params or AdamW step.
+ *   - Workers dispatched in one window share one snapshot slot, and a slot is recycled when its last
+ *     worker has been dispatched anew, so `base` is valid only until the next dispatch of ANY worker.
+ * So: call the accessor again after every alsgd_pull / alsgd_arrive before touching delta, p or base;
+ * writes through `p` are picked up by the next arrival or AdamW step of that worker.  A caller that
+ * must hold the pointers creates the context with ALSGD_CFG_STABLE_PTRS, which makes all of them
+ * permanent at the cost stated there. */
 int alsgd_state_ptrs(alsgd_ctx* ctx, alsgd_ptrs* out);
 int alsgd_worker_state_ptrs(alsgd_ctx* ctx, uint32_t worker, alsgd_worker_ptrs* out);
 
@@ -235,8 +263,16 @@ int alsgd_state_bytes(alsgd_ctx* ctx, uint64_t* bytes_out);
 int alsgd_export_state(alsgd_ctx* ctx, void* host_dst, uint64_t bytes);
 int alsgd_import_state(alsgd_ctx* ctx, const void* host_src, uint64_t bytes);
 
-/* Wait for the context's stream. */
+/* Wait for the context's stream.  In the debug build of the library (libalsgd_dbg.so, compiled with
+ * -DALSGD_DEBUG_BOUNDS: every kernel access to an arena-owned vector is checked against the arena's byte range
+ * and its alignment, an offending access is skipped and recorded instead of faulting) it then reads the
+ * record and returns ALSGD_E_BOUNDS if any access was refused since alsgd_init; the record is sticky. */
 int alsgd_sync(alsgd_ctx* ctx);
+
+/* Debug build: device address of the record alsgd_sync reads (one uint32, a bit per kind of vector: theta 1,
+ * Delta 2, m 4, worker parameters 8, snapshots 16, re-seed targets 32, AdamW p/m/v 64/128/256, replica 512), so
+ * that a caller can read or clear it.  Normal build: ALSGD_E_UNSUPPORTED and *word_out = NULL. */
+int alsgd_debug_word_ptr(alsgd_ctx* ctx, uint32_t** word_out);
 
 /* cudaError_t of the most recent failed CUDA call of this context (0 if none). */
 int alsgd_last_cuda_error(alsgd_ctx* ctx);

@@ -13,10 +13,10 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libalsgd.so")
 
-OK, E_ARG, E_RANGE, E_STATE, E_CUDA, E_NOMEM, E_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
+OK, E_ARG, E_RANGE, E_STATE, E_CUDA, E_NOMEM, E_UNSUPPORTED, E_BOUNDS = 0, -1, -2, -3, -4, -5, -6, -7
 TENSOR_DECAY = 1
 PG_DISPATCH, PG_CURRENT = 0, 1
-CFG_REPLICA_BF16, CFG_GRAD_STAGING, CFG_OUTER_BUFFERED = 1, 2, 4
+CFG_REPLICA_BF16, CFG_GRAD_STAGING, CFG_OUTER_BUFFERED, CFG_OUTER_SGDM, CFG_STABLE_PTRS = 1, 2, 4, 8, 16
 STALE_NONE, STALE_POLY, STALE_POLY_THRES = 0, 1, 2
 ARRIVE_RESEED, ARRIVE_NORM, ARRIVE_NANCHECK = 1, 2, 4
 
@@ -84,6 +84,7 @@ SIGNATURES = {
     "alsgd_export_state": (C.c_int, [_vp, _vp, C.c_uint64]),
     "alsgd_import_state": (C.c_int, [_vp, _vp, C.c_uint64]),
     "alsgd_sync": (C.c_int, [_vp]),
+    "alsgd_debug_word_ptr": (C.c_int, [_vp, C.POINTER(_vp)]),
     "alsgd_last_cuda_error": (C.c_int, [_vp]),
     "alsgd_dylu_steps": (C.c_int, [_f64p, C.c_uint32, C.c_uint32, _u32p]),
     "alsgd_shard_probs": (C.c_int, [_f64p, _f64p, C.c_uint32, _f64p]),

@@ -81,7 +81,9 @@ bool valid_cfg(const alsgd_config* c) {
     if (!c) return false;
     if (c->n_workers == 0 || c->N == 0) return false;
     if (c->pg_base != ALSGD_PG_DISPATCH && c->pg_base != ALSGD_PG_CURRENT) return false;
-    if (c->flags & ~(ALSGD_CFG_REPLICA_BF16 | ALSGD_CFG_GRAD_STAGING | ALSGD_CFG_OUTER_BUFFERED)) return false;
+    if (c->flags & ~(ALSGD_CFG_REPLICA_BF16 | ALSGD_CFG_GRAD_STAGING | ALSGD_CFG_OUTER_BUFFERED | ALSGD_CFG_OUTER_SGDM |
+                     ALSGD_CFG_STABLE_PTRS)) return false;
+    if ((c->flags & ALSGD_CFG_OUTER_BUFFERED) && (c->flags & ALSGD_CFG_OUTER_SGDM)) return false;
     if (!(c->beta >= 0.0f && c->beta < 1.0f)) return false;
     if (!std::isfinite(c->outer_lr)) return false;
     if (!(c->c >= 0.0f && (double)c->c * (double)c->N <= 1.0 + 1e-6)) return false;
@@ -96,7 +98,6 @@ struct alsgd_ctx {
     alsgd_config cfg;
     uint64_t P = 0;
     cudaStream_t stream = nullptr;
-    LaunchCfg lc{};
     // device slices
     uint64_t* seg_end = nullptr;
     uint32_t* seg_decay = nullptr;
@@ -104,6 +105,7 @@ struct alsgd_ctx {
     double* gnorm2 = nullptr;
     double* diag_partial = nullptr;
     unsigned int* nonfinite = nullptr;
+    unsigned int* guard_word = nullptr;   // debug build: violations recorded by the kernels' bounds checks
     float* theta = nullptr;
     float* mom = nullptr;
     float* delta = nullptr;
@@ -125,6 +127,10 @@ struct alsgd_ctx {
     // scalars of Algorithm 3, each rounded to fp32 once
     float inv_n = 0, cb = 0, cn = 0;
     int last_cuda = 0;
+    // Set when a call failed after some of its launches were already enqueued: the device state is then
+    // ahead of the host bookkeeping, and every later state-changing call is refused.
+    bool poisoned = false;
+    uintptr_t arena_lo = 0, arena_hi = 0;
 };
 
 namespace {
@@ -137,11 +143,12 @@ uint64_t carve(alsgd_ctx* c, void* arena, uint64_t P, const alsgd_config& cfg, u
     double* gn = k.take<double>(kMaxArrivals);
     double* gpart = k.take<double>(diag_partial_count(P));
     unsigned int* nf = k.take<unsigned int>(kMaxArrivals);
+    unsigned int* gw = k.take<unsigned int>(1);
     float* theta = k.take<float>(P);
     float* mom = k.take<float>(P);
     float* delta = k.take<float>(P);
     if (c) {
-        c->seg_end = seg_end; c->seg_decay = seg_decay; c->gnorm2 = gn; c->diag_partial = gpart; c->nonfinite = nf;
+        c->seg_end = seg_end; c->seg_decay = seg_decay; c->gnorm2 = gn; c->diag_partial = gpart; c->nonfinite = nf; c->guard_word = gw;
         c->theta = theta; c->mom = mom; c->delta = delta;
         c->workers.assign(cfg.n_workers, Worker());
         c->slot_ptr.clear();
@@ -204,10 +211,32 @@ void release_host_resources(alsgd_ctx* c) {
         if (c->chunk_ready[i]) { cudaEventDestroy(c->chunk_ready[i]); c->chunk_ready[i] = nullptr; }
 }
 
-void fill_seed(ArriveArgs& a, uint32_t slot, const Worker& w, float* snapshot, bool have_snapshots) {
-    a.seed_p[slot] = have_snapshots ? nullptr : w.p;     // with snapshots the parameters are read from there
-    a.seed_base[slot] = snapshot;
-    a.seed_rep[slot] = w.rep;
+bool stable_ptrs(const alsgd_ctx* c) { return (c->cfg.flags & ALSGD_CFG_STABLE_PTRS) != 0; }
+
+// Re-seed target s of a launch.  Normally the window's snapshot is written once (by the first target that is
+// handed it) and the parameters are not stored at all: readers take the snapshot until something writes p.
+// With ALSGD_CFG_STABLE_PTRS every worker keeps its own snapshot slot and its parameters are written too.
+void fill_seed(const alsgd_ctx* c, ArriveArgs& a, uint32_t s, uint32_t worker, float* snapshot) {
+    const Worker& w = c->workers[worker];
+    const bool have_snapshots = !c->slot_ptr.empty();
+    if (stable_ptrs(c)) {
+        a.seed_p[s] = w.p;
+        a.seed_base[s] = have_snapshots ? c->slot_ptr[worker] : nullptr;
+    } else {
+        a.seed_p[s] = have_snapshots ? nullptr : w.p;
+        a.seed_base[s] = snapshot;
+    }
+    a.seed_rep[s] = w.rep;
+}
+
+void fill_guard(const alsgd_ctx* c, DebugGuard& g) {
+#ifdef ALSGD_DEBUG_BOUNDS
+    g.lo = c->arena_lo;
+    g.hi = c->arena_hi;
+    g.err = c->guard_word;
+#else
+    (void)c; (void)g;
+#endif
 }
 
 // Where the worker's current parameters are to be read from.
@@ -228,7 +257,7 @@ int materialize_params(alsgd_ctx* c, Worker& w) {
 // is taken against the running theta and no snapshots exist).  At most W - k other workers hold a
 // slot, so one of the W slots is always free.
 int pick_slot(const alsgd_ctx* c, const uint32_t* ids, uint32_t k) {
-    if (c->slot_ptr.empty()) return -1;
+    if (c->slot_ptr.empty() || stable_ptrs(c)) return -1;
     std::vector<uint32_t> ref(c->slot_ref);
     for (uint32_t j = 0; j < k; ++j) {
         const int s = c->workers[ids[j]].slot;
@@ -240,7 +269,7 @@ int pick_slot(const alsgd_ctx* c, const uint32_t* ids, uint32_t k) {
 }
 
 void commit_slot(alsgd_ctx* c, const uint32_t* ids, uint32_t k, int s) {
-    if (s < 0) return;
+    if (s < 0) return;                                   // no snapshots, or every worker keeps its own
     for (uint32_t j = 0; j < k; ++j) {
         Worker& w = c->workers[ids[j]];
         if (w.slot >= 0) --c->slot_ref[w.slot];
@@ -264,6 +293,7 @@ const char* alsgd_strerror(int status) {
         case ALSGD_E_CUDA: return "CUDA runtime error";
         case ALSGD_E_NOMEM: return "not enough memory";
         case ALSGD_E_UNSUPPORTED: return "unsupported";
+        case ALSGD_E_BOUNDS: return "a kernel access fell outside the arena (debug build)";
         default: return "unknown status";
     }
 }
@@ -304,6 +334,8 @@ int alsgd_init(alsgd_ctx** out, const alsgd_tensor_desc* tensors, uint32_t n, ui
     c->stream = static_cast<cudaStream_t>(cfg->stream);
     c->n_seg = (uint32_t)seg.end.size();
     carve(c, cfg->arena, P, *cfg, c->n_seg);
+    c->arena_lo = reinterpret_cast<uintptr_t>(cfg->arena);
+    c->arena_hi = c->arena_lo + need;
     // Scalars of Algorithm 3: evaluated in double from the fp32 inputs, rounded to fp32 once.
     c->inv_n = 1.0f / (float)cfg->N;
     c->cb = (float)(((double)1.0 - (double)cfg->c * (double)cfg->N + (double)cfg->c) * (double)cfg->beta);
@@ -313,15 +345,13 @@ int alsgd_init(alsgd_ctx** out, const alsgd_tensor_desc* tensors, uint32_t n, ui
     {
         DeviceGuard g(cfg->device);
         cudaError_t e = g.ok ? cudaSuccess : cudaErrorInvalidDevice;
-        int sms = 0;
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device);
-        c->lc.sm_count = sms;
         if (e == cudaSuccess) e = cudaMemcpyAsync(c->seg_end, seg.end.data(), sizeof(uint64_t) * c->n_seg, cudaMemcpyHostToDevice, c->stream);
         if (e == cudaSuccess) e = cudaMemcpyAsync(c->seg_decay, seg.decay.data(), sizeof(uint32_t) * c->n_seg, cudaMemcpyHostToDevice, c->stream);
         // The segment tables live in pageable host vectors that die with this scope.
         if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->gnorm2, 0, sizeof(double) * kMaxArrivals, c->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * kMaxArrivals, c->stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->guard_word, 0, sizeof(unsigned int), c->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->theta, 0, sizeof(float) * P, c->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->mom, 0, sizeof(float) * P, c->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->delta, 0, sizeof(float) * P, c->stream);
@@ -383,16 +413,18 @@ int alsgd_get_worker_params(alsgd_ctx* c, uint32_t worker, float* dst, int dst_i
 int alsgd_pull(alsgd_ctx* c, uint32_t worker) {
     if (!c) return ALSGD_E_ARG;
     if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
+    if (c->poisoned) return ALSGD_E_STATE;
     Worker& w = c->workers[worker];
     ArriveArgs a{};
     a.theta = c->theta;
     a.n = c->P;
     a.n_arr = 0;
     a.n_seed = 1;
+    fill_guard(c, a.guard);
     const int slot = pick_slot(c, &worker, 1);
-    fill_seed(a, 0, w, slot >= 0 ? c->slot_ptr[slot] : nullptr, slot >= 0);
+    fill_seed(c, a, 0, worker, slot >= 0 ? c->slot_ptr[slot] : nullptr);
     DeviceGuard g(c->cfg.device);
-    ALSGD_CUDA(c, launch_arrive(a, false, false, false, c->lc, c->stream));
+    ALSGD_CUDA(c, launch_arrive(a, false, false, false, c->stream));
     commit_slot(c, &worker, 1, slot);
     w.pull_tick = c->t;
     w.state = kDispatched;
@@ -407,11 +439,12 @@ int adamw_impl(alsgd_ctx* c, uint32_t worker, const void* grads, bool bf16, int 
     if (!c || !grads || step == 0) return ALSGD_E_ARG;
     if (worker >= c->cfg.n_workers) return ALSGD_E_RANGE;
     Worker& w = c->workers[worker];
-    if (w.state == kNever) return ALSGD_E_STATE;
+    if (w.state == kNever || c->poisoned) return ALSGD_E_STATE;
     if (!grads_is_device && !c->grad_stage) return ALSGD_E_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(grads) % 16) return ALSGD_E_ARG;
     DeviceGuard g(c->cfg.device);
     AdamArgs a{};
+    fill_guard(c, a.guard);
     a.rep = w.rep;
     a.seg_end = c->seg_end; a.seg_decay = c->seg_decay; a.n_seg = c->n_seg;
     a.b1 = c->cfg.adam_b1; a.b2 = c->cfg.adam_b2;
@@ -430,7 +463,7 @@ int adamw_impl(alsgd_ctx* c, uint32_t worker, const void* grads, bool bf16, int 
         a.g16 = bf16 ? static_cast<const uint16_t*>(gsrc) : nullptr;
         a.n = len;
         a.seg_base = lo;
-        return launch_adamw(a, c->lc, c->stream);
+        return launch_adamw(a, c->stream);
     };
     if (grads_is_device) {
         ALSGD_CUDA(c, launch_range(0, c->P, grads));
@@ -448,7 +481,11 @@ int adamw_impl(alsgd_ctx* c, uint32_t worker, const void* grads, bool bf16, int 
             ALSGD_CUDA(c, cudaMemcpyAsync(stage + lo * esz, src + lo * esz, len * esz, cudaMemcpyHostToDevice, c->copy_stream));
             ALSGD_CUDA(c, cudaEventRecord(c->chunk_ready[i], c->copy_stream));
             ALSGD_CUDA(c, cudaStreamWaitEvent(c->stream, c->chunk_ready[i], 0));
-            ALSGD_CUDA(c, launch_range(lo, len, stage + lo * esz));
+            const cudaError_t le = launch_range(lo, len, stage + lo * esz);
+            if (le != cudaSuccess) {
+                if (i > 0) c->poisoned = true;            // earlier pieces of this step are already enqueued
+                return cuda_fail(c, le);
+            }
         }
     }
     w.p_in_snapshot = false;
@@ -500,11 +537,14 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
     }
     for (uint32_t j = 0; j < k; ++j)
         if (c->workers[ids[j]].state != kDispatched) return ALSGD_E_STATE;
+    if (c->poisoned) return ALSGD_E_STATE;
 
     const bool diag = (flags & (ALSGD_ARRIVE_NORM | ALSGD_ARRIVE_NANCHECK)) != 0;
     const bool reseed = (flags & ALSGD_ARRIVE_RESEED) != 0;
     const bool current = c->cfg.pg_base == ALSGD_PG_CURRENT;
-    const bool buffered = (c->cfg.flags & ALSGD_CFG_OUTER_BUFFERED) != 0;
+    const bool sgdm = (c->cfg.flags & ALSGD_CFG_OUTER_SGDM) != 0;
+    const bool buffered = sgdm || (c->cfg.flags & ALSGD_CFG_OUTER_BUFFERED) != 0;
+    const bool stable = stable_ptrs(c);
     const uint32_t N = c->cfg.N;
     const uint32_t rule = opts ? opts->staleness_rule : ALSGD_STALE_NONE;
     const float dc_lambda = opts ? opts->dc_lambda : 0.0f;
@@ -539,6 +579,14 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
     const int new_slot = reseed ? pick_slot(c, ids, k) : -1;   // one snapshot for the whole window
     float* snapshot = new_slot >= 0 ? c->slot_ptr[new_slot] : nullptr;
     bool snapshot_written = false;
+    bool enqueued = false;       // a launch of this call is already on the stream
+    // A failure after the first launch leaves theta, Delta and m ahead of the bookkeeping: refuse later calls.
+    auto fail = [&](cudaError_t e) { if (enqueued) c->poisoned = true; return cuda_fail(c, e); };
+#define ALSGD_STEP(call)                                 \
+    do {                                                 \
+        cudaError_t e__ = (call);                        \
+        if (e__ != cudaSuccess) return fail(e__);        \
+    } while (0)
     for (uint32_t ch = 0; ch < n_chunks; ++ch) {
         const uint32_t j0 = ch * kMaxArrivals;
         const uint32_t kk = (ka - j0 < (uint32_t)kMaxArrivals) ? ka - j0 : (uint32_t)kMaxArrivals;
@@ -549,14 +597,18 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
         a.n_arr = kk;
         a.beta = c->cfg.beta; a.eps = c->cfg.outer_lr; a.inv_n = c->inv_n; a.cb = c->cb; a.cn = c->cn;
         a.dc_lambda = dc_lambda;
-        a.beta2 = c->cfg.beta * c->cfg.beta;
-        a.one_plus_beta = 1.0f + c->cfg.beta;
+        // weights of the buffered step: Eq. 4 (beta^2, 1 + beta) or SGD Momentum (beta, 1)
+        a.beta2 = sgdm ? c->cfg.beta : c->cfg.beta * c->cfg.beta;
+        a.one_plus_beta = sgdm ? 1.0f : 1.0f + c->cfg.beta;
+        fill_guard(c, a.guard);
         bool any_boundary = false, last_boundary = false;
+        a.shared_base = current ? 0u : 1u;
         for (uint32_t j = 0; j < kk; ++j) {
             const uint32_t src = active[j0 + j];
             const Worker& w = c->workers[ids[src]];
             a.p[j] = params_of(w);
             a.base[j] = w.base;
+            if (a.base[j] != a.base[0]) a.shared_base = 0u;
             a.w[j] = plan[src].weight;
             const bool b = ((plan[src].tick + 1) % N) == 0;          // Algorithm 3's boundary test
             if (b) { a.boundary_mask |= 1u << j; any_boundary = true; }
@@ -564,7 +616,7 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
         }
         for (uint32_t j = kk; j < (uint32_t)kMaxArrivals; ++j) a.w[j] = 1.0f;
         if (delta_zero) a.flags |= kDeltaZeroIn;
-        if (last_boundary) a.flags |= kDeltaSkipStore;
+        if (last_boundary && !stable) a.flags |= kDeltaSkipStore;
         if (buffered) {
             a.flags |= kBuffered;
             if (!any_boundary) a.flags |= kSkipThetaStore;
@@ -575,25 +627,26 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
         if (any_boundary) a.flags |= kReadM | kWriteM;
         if (reseed && ch + 1 == n_chunks) {               // the final theta exists only in the last pass
             const uint32_t ns = k < (uint32_t)kMaxSeeds ? k : (uint32_t)kMaxSeeds;
-            for (uint32_t s = 0; s < ns; ++s) fill_seed(a, s, c->workers[ids[k - ns + s]], s == 0 ? snapshot : nullptr, snapshot != nullptr);
+            for (uint32_t s = 0; s < ns; ++s) fill_seed(c, a, s, ids[k - ns + s], s == 0 ? snapshot : nullptr);
             a.n_seed = ns;
             seeded = ns;
             snapshot_written = true;
         }
         if (diag) {
-            ALSGD_CUDA(c, cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * kMaxArrivals, c->stream));
+            ALSGD_STEP(cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * kMaxArrivals, c->stream));
         }
-        ALSGD_CUDA(c, launch_arrive(a, current, diag, extended, c->lc, c->stream));
+        ALSGD_STEP(launch_arrive(a, current, diag, extended, c->stream));
+        enqueued = true;
         if (diag && info) {
             double nb[kMaxArrivals];
             unsigned int fb[kMaxArrivals];
-            ALSGD_CUDA(c, cudaMemcpyAsync(nb, c->gnorm2, sizeof(double) * kk, cudaMemcpyDeviceToHost, c->stream));
-            ALSGD_CUDA(c, cudaMemcpyAsync(fb, c->nonfinite, sizeof(unsigned int) * kk, cudaMemcpyDeviceToHost, c->stream));
-            ALSGD_CUDA(c, cudaStreamSynchronize(c->stream));
+            ALSGD_STEP(cudaMemcpyAsync(nb, c->gnorm2, sizeof(double) * kk, cudaMemcpyDeviceToHost, c->stream));
+            ALSGD_STEP(cudaMemcpyAsync(fb, c->nonfinite, sizeof(unsigned int) * kk, cudaMemcpyDeviceToHost, c->stream));
+            ALSGD_STEP(cudaStreamSynchronize(c->stream));
             for (uint32_t j = 0; j < kk; ++j) { norms[active[j0 + j]] = nb[j]; bads[active[j0 + j]] = fb[j]; }
         }
         delta_zero = last_boundary;
-        delta_stored = !last_boundary;
+        delta_stored = !last_boundary || stable;
     }
     // Workers the arrival launches did not re-seed (a batch larger than one launch, or nothing but
     // discarded updates): the same final theta through standalone pulls.
@@ -603,14 +656,17 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
             const uint32_t ns = left < (uint32_t)kMaxSeeds ? left : (uint32_t)kMaxSeeds;
             ArriveArgs a{};
             a.theta = c->theta; a.n = c->P; a.n_seed = ns;
+            fill_guard(c, a.guard);
             for (uint32_t s = 0; s < ns; ++s) {
-                fill_seed(a, s, c->workers[ids[at + s]], snapshot_written ? nullptr : snapshot, snapshot != nullptr);
+                fill_seed(c, a, s, ids[at + s], snapshot_written ? nullptr : snapshot);
                 snapshot_written = true;
             }
-            ALSGD_CUDA(c, launch_arrive(a, false, false, false, c->lc, c->stream));
+            ALSGD_STEP(launch_arrive(a, false, false, false, c->stream));
+            enqueued = true;
             at += ns; left -= ns;
         }
     }
+#undef ALSGD_STEP
 
     // ---- commit bookkeeping
     if (info) {
@@ -804,6 +860,7 @@ int alsgd_import_state(alsgd_ctx* c, const void* host_src, uint64_t bytes) {
     c->t = h.t;
     c->delta_zero = h.delta_zero != 0;
     c->delta_stored = true;
+    c->poisoned = false;                                        // the whole state was replaced
     for (uint32_t w = 0; w < c->cfg.n_workers; ++w) {
         c->workers[w].pull_tick = iw[w].pull_tick;
         c->workers[w].state = (WorkerState)iw[w].state;
@@ -815,7 +872,24 @@ int alsgd_sync(alsgd_ctx* c) {
     if (!c) return ALSGD_E_ARG;
     DeviceGuard g(c->cfg.device);
     ALSGD_CUDA(c, cudaStreamSynchronize(c->stream));
+#ifdef ALSGD_DEBUG_BOUNDS
+    unsigned int word = 0;
+    ALSGD_CUDA(c, cudaMemcpyAsync(&word, c->guard_word, sizeof(word), cudaMemcpyDeviceToHost, c->stream));
+    ALSGD_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (word) return ALSGD_E_BOUNDS;
+#endif
     return ALSGD_OK;
+}
+
+int alsgd_debug_word_ptr(alsgd_ctx* c, uint32_t** word_out) {
+    if (!c || !word_out) return ALSGD_E_ARG;
+#ifdef ALSGD_DEBUG_BOUNDS
+    *word_out = c->guard_word;
+    return ALSGD_OK;
+#else
+    *word_out = nullptr;
+    return ALSGD_E_UNSUPPORTED;
+#endif
 }
 
 int alsgd_last_cuda_error(alsgd_ctx* c) { return c ? c->last_cuda : 0; }

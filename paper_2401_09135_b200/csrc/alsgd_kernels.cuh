@@ -19,6 +19,17 @@ enum : uint32_t {
     kSkipThetaStore = 128u // theta is unchanged by this launch (buffered, no boundary): do not write it
 };
 
+// Debug build only (-DALSGD_DEBUG_BOUNDS): the byte range every arena-owned access must stay in and the
+// word that records violations.  Empty in the normal build.
+#ifdef ALSGD_DEBUG_BOUNDS
+struct DebugGuard {
+    uintptr_t lo = 0, hi = 0;   // [lo, hi): the arena
+    unsigned int* err = nullptr;
+};
+#else
+struct DebugGuard {};
+#endif
+
 // One batch of arrivals of Algorithm 3 plus the re-seed of the workers that are dispatched again.
 struct ArriveArgs {
     float* theta;
@@ -41,7 +52,10 @@ struct ArriveArgs {
     // extended path only (weights, delay compensation, buffered outer step)
     float w[kMaxArrivals];            // staleness weights (1 = none)
     float dc_lambda;
-    float beta2, one_plus_beta;       // beta*beta and 1+beta, each one fp32 operation
+    float beta2, one_plus_beta;       // momentum and gradient weights of the buffered step: beta*beta and 1+beta
+                                      // (Eq. 4), or beta and 1 (SGD Momentum); each one fp32 operation
+    uint32_t shared_base;             // 1: every arrival was dispatched with the snapshot base[0]
+    DebugGuard guard;
 };
 
 struct AdamArgs {
@@ -58,16 +72,13 @@ struct AdamArgs {
     uint64_t n;                // elements in this launch
     uint64_t seg_base;         // flat index of this launch's first element (segment ends are flat indices)
     float b1, b2, omb1, omb2, bc1, bc2, eps, lr, wd;
-};
-
-struct LaunchCfg {
-    int sm_count;
+    DebugGuard guard;
 };
 
 // Entries of ArriveArgs::diag_partial needed for a vector of n elements (any batch size).
 uint64_t diag_partial_count(uint64_t n);
 
-cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, bool extended, const LaunchCfg& lc, cudaStream_t s);
-cudaError_t launch_adamw(const AdamArgs& a, const LaunchCfg& lc, cudaStream_t s);
+cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, bool extended, cudaStream_t s);
+cudaError_t launch_adamw(const AdamArgs& a, cudaStream_t s);
 
 }  // namespace alsgd
