@@ -274,6 +274,12 @@ int alsgd_sync(alsgd_ctx* ctx);
  * that a caller can read or clear it.  Normal build: ALSGD_E_UNSUPPORTED and *word_out = NULL. */
 int alsgd_debug_word_ptr(alsgd_ctx* ctx, uint32_t** word_out);
 
+/* Debug build: from now on treat only the first `bytes` of the arena as in range (0 = the whole arena again), so
+ * that the checks can be seen working without any access leaving the arena: accesses to the slices behind the
+ * limit are refused and recorded although the memory is the caller's own.  ALSGD_E_ARG if bytes exceeds the
+ * arena.  Normal build: ALSGD_E_UNSUPPORTED. */
+int alsgd_debug_guard_limit(alsgd_ctx* ctx, uint64_t bytes);
+
 /* cudaError_t of the most recent failed CUDA call of this context (0 if none). */
 int alsgd_last_cuda_error(alsgd_ctx* ctx);
 

@@ -85,6 +85,7 @@ SIGNATURES = {
     "alsgd_import_state": (C.c_int, [_vp, _vp, C.c_uint64]),
     "alsgd_sync": (C.c_int, [_vp]),
     "alsgd_debug_word_ptr": (C.c_int, [_vp, C.POINTER(_vp)]),
+    "alsgd_debug_guard_limit": (C.c_int, [_vp, C.c_uint64]),
     "alsgd_last_cuda_error": (C.c_int, [_vp]),
     "alsgd_dylu_steps": (C.c_int, [_f64p, C.c_uint32, C.c_uint32, _u32p]),
     "alsgd_shard_probs": (C.c_int, [_f64p, _f64p, C.c_uint32, _f64p]),
@@ -99,6 +100,17 @@ SIGNATURES = {
 STATIC_MAX_ELEMS = 1 << 27
 
 _lib = None
+_variant = "main"
+
+
+def use_debug_library(on: bool = True):
+    """Route every later call through libalsgd_dbg.so (kernels with bounds checks; alsgd_sync reports refused
+    accesses) instead of libalsgd.so.  Must be chosen before the first call that loads a library."""
+    global _variant
+    want = "debug" if on else "main"
+    if _lib is not None and want != _variant:
+        raise RuntimeError("a library is already loaded in this process")
+    _variant = want
 
 
 class AlsgdError(RuntimeError):
@@ -119,11 +131,12 @@ def lib():
     global _lib
     if _lib is None:
         from . import build as _build
-        if _build.needs_build():
-            _build.build()
-        if not os.path.exists(LIB_PATH):
-            raise RuntimeError(f"{LIB_PATH} is missing: the CUDA library is required, there is no fallback")
-        L = C.CDLL(LIB_PATH)
+        if _build.needs_build(_variant):
+            _build.build(targets=(_variant,))
+        path = LIB_PATH if _variant == "main" else _build.LIB_DBG
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: the CUDA library is required, there is no fallback")
+        L = C.CDLL(path)
         for name, (res, args) in SIGNATURES.items():
             fn = getattr(L, name)      # AttributeError if the library does not export a declared symbol
             fn.restype, fn.argtypes = res, args
@@ -218,7 +231,7 @@ class Context:
 
     def __init__(self, tensors, n_workers, N, beta, outer_lr, c=0.0, pg_base=PG_DISPATCH,
                  adam=(0.9, 0.95, 1e-8, 0.1), replica=True, grad_staging=False, align_elems=128,
-                 device=0, stream=None, buffered=False):
+                 device=0, stream=None, buffered=False, sgdm=False, stable_ptrs=False):
         import torch
         self.torch = torch
         if not torch.cuda.is_available():
@@ -230,7 +243,8 @@ class Context:
         cfg = Config()
         cfg.n_workers, cfg.N, cfg.pg_base = int(n_workers), int(N), int(pg_base)
         cfg.flags = ((CFG_REPLICA_BF16 if replica else 0) | (CFG_GRAD_STAGING if grad_staging else 0)
-                     | (CFG_OUTER_BUFFERED if buffered else 0))
+                     | (CFG_OUTER_BUFFERED if buffered else 0) | (CFG_OUTER_SGDM if sgdm else 0)
+                     | (CFG_STABLE_PTRS if stable_ptrs else 0))
         cfg.beta, cfg.outer_lr, cfg.c = float(beta), float(outer_lr), float(c)
         cfg.adam_b1, cfg.adam_b2, cfg.adam_eps, cfg.adam_wd = [float(x) for x in adam]
         cfg.device = device
@@ -358,6 +372,12 @@ class Context:
 
     def alsgd_sync(self):
         _check(lib().alsgd_sync(self._h), "alsgd_sync", self._h)
+
+    def alsgd_debug_word_ptr(self):
+        """Device address of the debug build's violation record (raises E_UNSUPPORTED on the normal build)."""
+        out = _vp()
+        _check(lib().alsgd_debug_word_ptr(self._h, C.byref(out)), "alsgd_debug_word_ptr", self._h)
+        return int(out.value)
 
     def raw(self, name, *args):
         """Call an ABI function on this context and return its status without raising."""

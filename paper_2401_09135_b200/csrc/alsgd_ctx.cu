@@ -335,7 +335,7 @@ int alsgd_init(alsgd_ctx** out, const alsgd_tensor_desc* tensors, uint32_t n, ui
     c->n_seg = (uint32_t)seg.end.size();
     carve(c, cfg->arena, P, *cfg, c->n_seg);
     c->arena_lo = reinterpret_cast<uintptr_t>(cfg->arena);
-    c->arena_hi = c->arena_lo + need;
+    c->arena_hi = c->arena_lo + cfg->arena_bytes;
     // Scalars of Algorithm 3: evaluated in double from the fp32 inputs, rounded to fp32 once.
     c->inv_n = 1.0f / (float)cfg->N;
     c->cb = (float)(((double)1.0 - (double)cfg->c * (double)cfg->N + (double)cfg->c) * (double)cfg->beta);
@@ -879,6 +879,19 @@ int alsgd_sync(alsgd_ctx* c) {
     if (word) return ALSGD_E_BOUNDS;
 #endif
     return ALSGD_OK;
+}
+
+int alsgd_debug_guard_limit(alsgd_ctx* c, uint64_t bytes) {
+    if (!c) return ALSGD_E_ARG;
+#ifdef ALSGD_DEBUG_BOUNDS
+    const uint64_t whole = c->cfg.arena_bytes;
+    if (bytes > whole) return ALSGD_E_ARG;
+    c->arena_hi = c->arena_lo + (bytes ? bytes : whole);
+    return ALSGD_OK;
+#else
+    (void)bytes;
+    return ALSGD_E_UNSUPPORTED;
+#endif
 }
 
 int alsgd_debug_word_ptr(alsgd_ctx* c, uint32_t** word_out) {

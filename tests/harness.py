@@ -46,14 +46,15 @@ def assert_fp32(name, got, ref, strict=True):
 class Pair:
     def __init__(self, tensors, n_workers, N, beta, outer_lr, c=0.0, pg_current=False, replica=True,
                  adam=(0.9, 0.95, 1e-8, 0.1), align=128, n_sample=None, grad_staging=False, strict=True,
-                 buffered=False):
+                 buffered=False, sgdm=False, stable_ptrs=False):
         self.tensors = tensors
         self.W = n_workers
         self.strict = strict
         self.ctx = B.Context(tensors, n_workers, N, beta, outer_lr, c=c,
                              pg_base=B.PG_CURRENT if pg_current else B.PG_DISPATCH, adam=adam, replica=replica,
-                             grad_staging=grad_staging, align_elems=align, buffered=buffered)
-        self.buffered = buffered
+                             grad_staging=grad_staging, align_elems=align, buffered=buffered, sgdm=sgdm,
+                             stable_ptrs=stable_ptrs)
+        self.buffered = oracle.OUTER_SGDM if sgdm else (oracle.OUTER_BUFFERED if buffered else oracle.OUTER_DN)
         self.P, self.offsets = self.ctx.P, self.ctx.offsets
         o_offs, o_P = oracle.layout_offsets([t.numel for t in tensors], align)
         assert (o_P, o_offs) == (self.P, self.offsets)

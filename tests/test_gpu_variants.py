@@ -137,3 +137,28 @@ def test_arrive_ex_argument_errors():
     assert ctx.raw("alsgd_arrive_ex", ids, 1, 0, None, None) == B.OK       # NULL opts == alsgd_arrive
     assert ctx.alsgd_counters()[0] == 1
     ctx.close()
+
+
+@pytest.mark.parametrize("N", [1, 3, 4])
+def test_sgd_momentum_outer_step(N):
+    """ALSGD_CFG_OUTER_SGDM: the heavy-ball step on the buffer mean at every N-th arrival (N = 1: at every arrival)."""
+    pair = Pair(synth.ragged_tensors(), 5, N, 0.9, 0.7, align=8, sgdm=True)
+    start(pair)
+    for b, ids in enumerate(BATCHES):
+        perturb_all(pair, ids, b)
+        theta_before = pair.ctx.alsgd_state_ptrs()[0].clone()
+        info = pair.arrive(ids, reseed=True, norm=True, weights=[0.5] * len(ids) if b == 3 else None)
+        pair.check_all(f"batch {b}")
+        if not any(i["boundary"] for i in info):
+            assert torch.equal(theta_before, pair.ctx.alsgd_state_ptrs()[0])
+    pair.close()
+
+
+def test_outer_modes_exclude_each_other():
+    cfg_flags = B.CFG_OUTER_BUFFERED | B.CFG_OUTER_SGDM
+    tab = B.tensor_table(synth.flat_tensors(64))
+    cfg = B.Config()
+    cfg.n_workers, cfg.N, cfg.flags, cfg.beta, cfg.outer_lr = 1, 1, cfg_flags, 0.9, 0.7
+    cfg.adam_b1, cfg.adam_b2, cfg.adam_eps, cfg.adam_wd = 0.9, 0.95, 1e-8, 0.1
+    n = C.c_uint64()
+    assert B.lib().alsgd_arena_bytes(tab, 1, 1, C.byref(cfg), C.byref(n)) == B.E_ARG
