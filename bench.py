@@ -8,7 +8,11 @@ Delayed-Nesterov arrival with the fused re-seed.  Each kernel launch streams the
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-Prints ONE JSON line on rank 0.
+Prints ONE JSON line on rank 0.  At N = 1 the line also carries the reported figures of the other configurations
+(`ksweep`: arrival batches k = 1, 2, 4, 8 with 8 resident workers; `layouts`: per-kernel throughput on the 23M /
+60M / 110M / 150M layouts), measured after the timed region, and the oracle timed on one and on all host cores.
+Further modes: --ksweep, --layouts, --cpu-kernels, --shape-sweep (launch-shape benchmark), --profile-case
+(small fixed cases for profiler captures).
 """
 import argparse
 import hashlib
@@ -131,6 +135,17 @@ def build_schedule(n_arrivals):
     return steps, order[:n_arrivals]
 
 
+def oracle_schedule(n_arrivals):
+    """The same schedule from the oracle alone (Eq. 6 and Algorithms 2 + 5 as the oracle states them), so that
+    the reference arm needs nothing of the CUDA library."""
+    import oracle
+    from paper_2401_09135_b200 import synth
+    steps = oracle.dylu(SPEEDS, H)
+    dur = synth.job_durations(SPEEDS, steps, n_arrivals + 2, synth.SEED + 7)
+    workers, _, _ = oracle.schedule(dur, steps, 0.0, 10 ** 18, n_arrivals)
+    return steps, workers
+
+
 # ----------------------------------------------------------------------------------------------------
 # reference arm: the CPU oracle, as it stands, on the host cores
 # ----------------------------------------------------------------------------------------------------
@@ -166,12 +181,39 @@ def run_oracle(n_elems, order, steps, warmup, timed):
     return n_elems * passes / dt, dt, passes
 
 
+def run_oracle_all_cores(n_elems, w, n_inner, threads):
+    """One step of the same path with the oracle's scalar loops range-split over `threads` host threads (exact:
+    the path is elementwise; the C functions release the interpreter lock)."""
+    import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
+    import oracle
+    from paper_2401_09135_b200 import synth
+    tensors = synth.layout_110m()
+    offs, P = oracle.layout_offsets([t.numel for t in tensors], 128)
+    mask = oracle.decay_mask([t.numel for t in tensors], [t.decay for t in tensors], offs, P)[:n_elems].copy()
+    z = lambda: np.zeros(n_elems, np.float32)
+    theta = synth.normal_vec(n_elems, 0.02, synth.SEED, synth.STREAM_THETA0)
+    m, D, p, base, am, av, rep = z(), z(), theta.copy(), theta.copy(), z(), z(), np.zeros(n_elems, np.uint16)
+    g = synth.normal_vec(n_elems, 1e-2, synth.SEED, synth.STREAM_GRAD)
+    cuts = [n_elems * i // threads for i in range(threads + 1)]
+    with ThreadPoolExecutor(threads) as ex:
+        def every(fn):
+            list(ex.map(lambda i: fn(cuts[i], cuts[i + 1]), range(threads)))
+        t0 = time.perf_counter()
+        for s in range(1, n_inner + 1):
+            every(lambda lo, hi: oracle.adamw(p, am, av, g, rep, mask, s, 1e-3, 0.9, 0.95, 1e-8, 0.1, lo=lo, hi=hi))
+        every(lambda lo, hi: oracle.dn_arrive(theta, m, D, base, p, 0, 4, 0.9, 0.7, lo=lo, hi=hi))
+        every(lambda lo, hi: oracle.reseed(theta, p, base, rep, lo=lo, hi=hi))
+        dt = time.perf_counter() - t0
+    return n_elems * (n_inner + 1) / dt, dt
+
+
 def main_reference(args, rank):
     if rank != 0:
         return
     import oracle
     oracle.build()
-    steps, order = build_schedule(args.warmup + args.steps)
+    steps, order = oracle_schedule(args.warmup + args.steps)
     n_elems = 1 << 22
     value, dt, passes = run_oracle(n_elems, order, steps, args.warmup, args.steps)
     sample = f"first {n_elems} elements of the layout, every step of the schedule (DyLU inner steps + arrival)"
@@ -338,34 +380,52 @@ def main_ours(args, rank, world, local_rank):
             "adamw_bf16_grads": {"avg_ms": adam16_ms, "bytes_per_param": 28, "achieved": 28 * P / (adam16_ms * 1e-3) / 1e9,
                                  "unit": "GB/s", "launches": 20, "note": "extra; not part of the timed steps"},
         }
+        for key, traffic in (("roofline", adam_traffic), ("roofline_arrive", arr_traffic)):
+            if traffic:           # the same launch on the DRAM bytes ncu counted (dirty L2 lines at kernel end are not in them)
+                r = line[key]
+                r["achieved_on_measured_traffic"] = traffic / (r["avg_ms"] * 1e-3) / 1e9
+                r["frac_of_nominal_8TBs_on_measured_traffic"] = r["achieved_on_measured_traffic"] / NOMINAL_HBM_GBS
+    ctx.alsgd_sync()
+    ctx.close()
+    del ctx, gpool
+    torch.cuda.empty_cache()
+    if rank == 0:
+        if world == 1 and not args.no_extras:
+            # the reported figures of the other configurations: arrival batches k = 1, 2, 4, 8 with 8 resident
+            # workers, and per-kernel throughput on the 23M / 60M / 110M / 150M layouts
+            line["ksweep"] = run_ksweep(args, local_rank)
+            line["layouts"] = run_layouts(args, local_rank)
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
             n_cpu = P // 8
             cpu_order = [order[0]]
             v, dt, p = run_oracle(n_cpu, cpu_order, steps, 0, 1)
-            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
-                                    "sample": f"first {n_cpu} elements (an eighth) of the layout, one step: {steps[cpu_order[0]]} inner AdamW steps + 1 arrival with re-seed"}
+            sample = f"first {n_cpu} elements (an eighth) of the layout, one step: {steps[cpu_order[0]]} inner AdamW steps + 1 arrival with re-seed"
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt, "sample": sample}
+            cores = os.cpu_count() or 1
+            vn, dtn = run_oracle_all_cores(n_cpu, cpu_order[0], steps[cpu_order[0]], cores)
+            line["cpu_baseline"]["all_cores"] = {"value": vn, "unit": UNIT, "cores": cores, "seconds": dtn,
+                                                 "how": "the oracle's scalar loops range-split over host threads, same sample"}
         print(json.dumps(line), flush=True)
-    ctx.close()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
 
 
-def main_ksweep(args):
+def run_ksweep(args, device=0):
     """Arrival-batch sweep on the 110M layout with 8 resident workers (N = 8): per k, each round is 8/k
     batches of k through the multi-arrival kernel with fused re-seed, then 10 AdamW steps per worker."""
     import torch
     from paper_2401_09135_b200 import binding as B, synth
-    torch.cuda.set_device(0)
+    torch.cuda.set_device(device)
     tensors = synth.layout_110m()
     W, N, inner = 8, 8, 10
     peak, which = measured_peak()
     out = []
     gpool = None
     for k in (1, 2, 4, 8):
-        ctx = B.Context(tensors, W, N, 0.9, 0.7)
+        ctx = B.Context(tensors, W, N, 0.9, 0.7, device=device)
         P = ctx.P
         if gpool is None:
             gpool = [torch.from_numpy(synth.normal_vec(P, 1e-2, synth.SEED, synth.STREAM_GRAD, sub=i)).cuda() for i in range(2)]
@@ -403,26 +463,33 @@ def main_ksweep(args):
                     "arrivals_per_s": W / (arr_ms * 1e-3), "adamw_ms_per_round": adam_ms,
                     "adamw_gbs": adam_bytes / adam_ms / 1e6, "adamw_frac": adam_bytes / adam_ms / 1e6 / peak,
                     "combined_gbs": (arr_bytes + adam_bytes) / (arr_ms + adam_ms) / 1e6,
-                    "combined_frac": (arr_bytes + adam_bytes) / (arr_ms + adam_ms) / 1e6 / peak})
+                    "combined_frac": (arr_bytes + adam_bytes) / (arr_ms + adam_ms) / 1e6 / peak,
+                    "arrival_frac_of_8TBs": arr_bytes / arr_ms / 1e6 / NOMINAL_HBM_GBS,
+                    "adamw_frac_of_8TBs": adam_bytes / adam_ms / 1e6 / NOMINAL_HBM_GBS})
+        ctx.alsgd_sync()
         ctx.close()
         del ctx
         torch.cuda.empty_cache()
-    print(json.dumps({"workload": "decoder-110M W=8 N=8 beta=0.9 outer_lr=0.7, k-sweep, 10 inner AdamW steps per worker per round",
-                      "peak_gbs": peak, "peak_source": f"of {which}", "unit": "GB/s", "rounds_timed": len(ev), "sweep": out}), flush=True)
+    return {"workload": "decoder-110M W=8 N=8 beta=0.9 outer_lr=0.7, k-sweep, 10 inner AdamW steps per worker per round",
+            "peak_gbs": peak, "peak_source": f"of {which}", "unit": "GB/s", "rounds_timed": len(ev), "sweep": out}
 
 
-def main_layouts(args):
+def main_ksweep(args):
+    print(json.dumps(run_ksweep(args)), flush=True)
+
+
+def run_layouts(args, device=0):
     """Per-kernel throughput on layouts shaped like the paper's 20M-150M decoder transformers (2 workers, N = 4):
     20 AdamW steps and 20 single arrivals with fused re-seed each, CUDA events, after 4 warm-up launches.
     Below ~30M elements one fp32 buffer fits in L2, so those rows are not HBM-roofline figures."""
     import torch
     from paper_2401_09135_b200 import binding as B, synth
-    torch.cuda.set_device(0)
+    torch.cuda.set_device(device)
     peak, which = measured_peak()
     out = []
     for name, tensors in (("23M (6L, d384, ff1536)", synth.layout_23m()), ("paper 60M (3L, h896, 16x64)", synth.layout_paper_60m()),
                           ("110M (12L, d768, ff3072)", synth.layout_110m()), ("paper 150M (12L, h896, 16x64)", synth.layout_paper_150m())):
-        ctx = B.Context(tensors, 2, 4, 0.9, 0.7)
+        ctx = B.Context(tensors, 2, 4, 0.9, 0.7, device=device)
         P = ctx.P
         ctx.alsgd_set_global(synth.theta0(tensors, ctx.offsets, P))
         g = [torch.from_numpy(synth.normal_vec(P, 1e-2, synth.SEED, synth.STREAM_GRAD, sub=i)).cuda() for i in range(2)]
@@ -460,9 +527,17 @@ def main_layouts(args):
             res[key] = {"ms": ms, "params_per_s": P / (ms * 1e-3), "gbs": bpp * P / (ms * 1e-3) / 1e9,
                         "frac_of_measured": bpp * P / (ms * 1e-3) / 1e9 / peak, "frac_of_8TBs": bpp * P / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS}
         out.append(res)
+        ctx.alsgd_sync()
         ctx.close(); del ctx, g
         torch.cuda.empty_cache()
-    print(json.dumps({"peak_gbs": peak, "peak_source": f"of {which}", "layouts": out}), flush=True)
+    return {"peak_gbs": peak, "peak_source": f"of {which}", "unit": "GB/s",
+            "note": "2 workers, N = 4; 20 AdamW steps and 20 single arrivals with fused re-seed per layout, CUDA events; "
+                    "one fp32 vector of the 23M layout (92 MB) fits in the 126 MB L2, so that row is no HBM roofline figure",
+            "layouts": out}
+
+
+def main_layouts(args):
+    print(json.dumps(run_layouts(args)), flush=True)
 
 
 def main_shape_sweep(args):
@@ -486,6 +561,64 @@ def main_shape_sweep(args):
             best[key] = r
     print(json.dumps({"elements": n, "reps": args.sweep_reps, "peak_gbs": peak, "peak_source": f"of {which}",
                       "unit": "GB/s on algorithmic bytes", "best": best, "rows": rows}), flush=True)
+
+
+def main_profile_case(args):
+    """Small fixed cases for profiler captures: a few launches of each kernel on vectors larger than L2 but only a
+    few GB on the device in total.
+      single   2 workers, N = 4, 48Mi elements (2.4 GB): 2 pulls, 3 AdamW steps per worker, then four times (AdamW
+               step, single arrival with fused re-seed) through one Delayed-Nesterov cycle (first / middle / middle /
+               boundary), one AdamW step per worker, one batch of two
+      batches  8 workers, N = 8, 32Mi elements (4.3 GB): pulls, one AdamW step each, two batches of 4, one AdamW step
+               each, one batch of 8 (all sharing one dispatch snapshot)
+      diag     the batches case with the squared-norm / non-finite diagnostics requested on every arrival"""
+    import torch
+    from paper_2401_09135_b200 import binding as B, synth
+    torch.cuda.set_device(0)
+    mode = args.profile_case
+    if mode in ("batches", "diag"):
+        flags = B.ARRIVE_RESEED | ((B.ARRIVE_NORM | B.ARRIVE_NANCHECK) if mode == "diag" else 0)
+        tensors = synth.flat_tensors(32 * 1024 * 1024)
+        W = 8
+        ctx = B.Context(tensors, W, 8, 0.9, 0.7)
+        ctx.alsgd_set_global(synth.theta0(tensors, ctx.offsets, ctx.P))
+        g = torch.from_numpy(synth.normal_vec(ctx.P, 1e-2, synth.SEED, synth.STREAM_GRAD)).cuda()
+        for w in range(W):
+            ctx.alsgd_pull(w)
+        for w in range(W):
+            ctx.alsgd_inner_adamw(w, g, 1, 1e-3)
+        ctx.alsgd_arrive([0, 1, 2, 3], flags, want_info=False)     # first of the cycle, one shared snapshot
+        ctx.alsgd_arrive([4, 5, 6, 7], flags, want_info=False)     # ends the cycle of N = 8 (boundary inside)
+        for w in range(W):
+            ctx.alsgd_inner_adamw(w, g, 2, 1e-3)
+        ctx.alsgd_arrive(list(range(W)), flags, want_info=False)   # whole cycle in one pass, two snapshots among the 8
+        for w in range(W):
+            ctx.alsgd_inner_adamw(w, g, 3, 1e-3)
+        ctx.alsgd_arrive(list(range(W)), flags, want_info=False)   # whole cycle in one pass, all 8 share one snapshot
+    else:
+        n = 48 * 1024 * 1024
+        tensors = [synth.Tensor("w0", n // 2, True, "matrix"), synth.Tensor("g0", 4096, False, "gain"),
+                   synth.Tensor("w1", n - n // 2 - 4096, True, "matrix")]
+        ctx = B.Context(tensors, 2, 4, 0.9, 0.7)
+        ctx.alsgd_set_global(synth.theta0(tensors, ctx.offsets, ctx.P))
+        g = torch.from_numpy(synth.normal_vec(ctx.P, 1e-2, synth.SEED, synth.STREAM_GRAD)).cuda()
+        for w in range(2):
+            ctx.alsgd_pull(w)
+        for w in range(2):
+            for st in range(1, 4):
+                ctx.alsgd_inner_adamw(w, g, st, 1e-3)
+        step = [3, 3]
+        for w in (0, 1, 0, 1):
+            step[w] += 1
+            ctx.alsgd_inner_adamw(w, g, step[w], 1e-3)
+            ctx.alsgd_arrive([w], B.ARRIVE_RESEED, want_info=False)
+        for w in range(2):
+            step[w] += 1
+            ctx.alsgd_inner_adamw(w, g, step[w], 1e-3)
+        ctx.alsgd_arrive([0, 1], B.ARRIVE_RESEED, want_info=False)
+    ctx.alsgd_sync()
+    print(f"profile case {mode} done: P={ctx.P}, t={ctx.alsgd_counters()[0]}")
+    ctx.close()
 
 
 def main_cpu_kernels(args):
@@ -538,9 +671,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the k-sweep and layout tables of the default line")
     ap.add_argument("--ksweep", action="store_true", help="arrival-batch sweep (k = 1, 2, 4, 8) with 8 resident workers")
     ap.add_argument("--layouts", action="store_true", help="per-kernel throughput on 23M / 60M / 110M / 150M layouts")
     ap.add_argument("--cpu-kernels", action="store_true", help="time the oracle's loops per kernel on the host cores")
+    ap.add_argument("--profile-case", choices=["single", "batches", "diag"], help="run a small fixed case for a profiler capture")
     ap.add_argument("--shape-sweep", action="store_true", help="time the launch shapes of libalsgd_sweep.so")
     ap.add_argument("--sweep-elems", type=int, default=109_549_056)
     ap.add_argument("--sweep-reps", type=int, default=10)
@@ -549,7 +684,9 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.shape_sweep:
+    if args.profile_case:
+        main_profile_case(args)
+    elif args.shape_sweep:
         main_shape_sweep(args)
     elif args.layouts:
         main_layouts(args)

@@ -355,7 +355,12 @@ int alsgd_sched_local_updates(alsgd_sched* s, uint64_t* t_local_out);
  *                   order (the same inputs give the same bits on every call)
  *   nonfinite_out   device, one uint32: 1 if any entry of start - p is NaN or Inf, else 0
  * The call only enqueues; the outputs are valid once the stream reaches them.  The first call on each
- * device looks up the array's device address; make that first call outside any stream capture.
+ * device looks up the array's device address; make that first call outside any stream capture.  With the
+ * CUDA runtime's default lazy module loading that first call is also the moment the device sets the array and
+ * this entry point's kernels aside, so a process that hands out all of its device memory should make one
+ * warm-up call (n = 4 on any two valid buffers is enough) at start-up, before it does so: afterwards no call
+ * needs anything more.  The looked-up address is cached per device ordinal for the life of the process and
+ * does not survive a reset of that device's primary context (cudaDeviceReset).
  * All calls on one device share the one array and it keeps the previous call's contents, so the call
  * clears what it accumulates into before use; two calls whose kernels can overlap on the GPU (other
  * streams, other threads) race on it and must be ordered by the caller.

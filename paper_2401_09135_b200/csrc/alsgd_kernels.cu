@@ -8,25 +8,29 @@ namespace {
 
 using namespace kern;
 
-// Launch shape per number of arrivals K and snapshot mode: float4 vectors per thread, threads per
-// block, packed two-lane arithmetic.  Chosen from the launch-shape benchmark (bench.py --shape-sweep)
-// on B200 at 110M elements.
+// Launch shape per number of arrivals K: float4 vectors per thread per stream, threads per block, packed
+// two-lane arithmetic.  From the launch-shape benchmark (bench.py --shape-sweep) on B200 at 110M elements:
+// every one-tile-per-block shape with at most ~20 vectors in flight per thread lands within 1 % of 6.8 TB/s
+// (the memory system's rate for these read/write mixes); what separates them is how they degrade once the
+// diagnostics or eight arrivals add registers and arithmetic.  One vector per thread keeps the registers low
+// at every K; with five or more arrivals 128-thread blocks pack more warps into the register file than
+// 256-thread blocks (K = 8 with diagnostics: 6.55 against 6.02 TB/s) and the packed arithmetic halves the
+// instruction count of the K-fold update (6.55 against 6.47 TB/s); at K <= 4 neither matters.
 struct Shape {
     int V, BLK;
     bool PK;
 };
-constexpr Shape arrive_shape(int K, int base) {
-    (void)base;
-    if (K <= 1) return {4, 256, false};
-    if (K <= 4) return {2, 256, false};
-    return {1, 256, false};
+constexpr Shape arrive_shape(int K) {
+    if (K == 0) return {4, 256, false};           // re-seed only: one read stream, up to three written
+    if (K <= 4) return {1, 256, false};
+    return {1, 128, true};
 }
-constexpr Shape kAdamShape = {2, 256, false};
-constexpr int kMinTileVecs = 256;                 // smallest BLK * V of any arrival shape: the most blocks a launch can have
+constexpr Shape kAdamShape = {1, 128, false};     // 6.82 TB/s; two vectors per thread in 256-thread blocks: 6.65-6.83
+constexpr int kMinTileVecs = 128;                 // smallest BLK * V of any arrival shape: the most blocks a launch can have
 
 template <int K, bool DIAG, int BASE, bool EXT>
 cudaError_t launch_arrive_k(const ArriveArgs& a, cudaStream_t s) {
-    constexpr Shape sh = arrive_shape(K, BASE);
+    constexpr Shape sh = arrive_shape(K);
     static_assert(sh.V * sh.BLK >= kMinTileVecs, "diag_partial_count assumes at least kMinTileVecs vectors per block");
     auto kern = arrive_kernel<K, sh.V, sh.BLK, 1, DIAG, BASE, EXT, false, sh.PK>;
     unsigned grid = 1;

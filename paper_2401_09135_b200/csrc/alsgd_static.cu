@@ -34,7 +34,9 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 std::mutex g_setup_mutex;
 void* g_scratch_addr[kMaxDevices] = {};                    // per device ordinal, filled on first use
 
-// Device address of the array on `device`, which must be the current device.
+// Device address of the array on `device`, which must be the current device.  The first call per device is
+// also what makes a lazily loading runtime place this module (the array and the two kernels) on the device.
+// The cached address belongs to the device's primary context and is stale after a reset of that context.
 cudaError_t scratch_address(int device, void** out) {
     std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (!g_scratch_addr[device]) {

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2401_09135_b200 import binding as B
 from paper_2401_09135_b200 import synth
 
@@ -41,12 +42,14 @@ def test_static_entry_point_matches_arrive_diagnostics_twice(P):
         assert static_norm(v["base"], v["p"], ctx.P, out_norm, out_flag) == B.OK
         repeat = torch.empty_like(out_norm)
         assert static_norm(v["base"], v["p"], ctx.P, repeat, out_flag) == B.OK
+        o_norm, o_flag = oracle.pg_norm2(v["base"].cpu().numpy(), v["base"].cpu().numpy(), v["p"].cpu().numpy())
         info = ctx.alsgd_arrive([w], B.ARRIVE_NORM | B.ARRIVE_NANCHECK)[0]
         torch.cuda.synchronize()
-        assert int(out_flag.item()) == info["nonfinite"] == call
+        assert int(out_flag.item()) == info["nonfinite"] == o_flag == call
         if call == 0:
             got, ref = float(out_norm.item()), info["gnorm2"]
             assert ref > 0 and abs(got - ref) <= 1e-6 * ref          # same tolerance as the norm parity tests
+            assert abs(got - o_norm) <= 1e-6 * o_norm                # and directly against the CPU oracle's double sum
             assert float(repeat.item()) == got                       # fixed summation order: same bits
     ctx.close()
 
@@ -66,3 +69,33 @@ def test_static_entry_point_limits_and_arguments():
     assert L.alsgd_pg_norm_static(x.data_ptr(), x.data_ptr(), 4096, 0, s, n64.data_ptr(), f32.data_ptr()) == B.OK
     torch.cuda.synchronize()
     assert float(n64.item()) == 0.0 and int(f32.item()) == 0
+
+
+@pytest.mark.parametrize("n", [B.STATIC_MAX_ELEMS, B.STATIC_MAX_ELEMS - 3])
+def test_static_entry_point_at_its_size_limit(n):
+    """The largest accepted vector uses every slot of the fixed working memory (n = limit), and limit - 3 ends in a
+    ragged tile.  Every pseudo-gradient entry is +-2^-10, so the exact sum is n * 2^-20 and every partial sum is
+    exact in double: the result must match to the last bit.  1 GiB of inputs."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 3 * (1 << 30):
+        pytest.skip("needs 3 GiB of free device memory")
+    start = torch.ones(n, dtype=torch.float32, device="cuda")
+    p = torch.ones(n, dtype=torch.float32, device="cuda")
+    p[0::2] += 2.0 ** -10
+    p[1::2] -= 2.0 ** -10
+    out_norm = torch.full((1,), -1.0, dtype=torch.float64, device="cuda")
+    out_flag = torch.full((1,), 7, dtype=torch.int32, device="cuda")
+    for _ in range(2):
+        assert static_norm(start, p, n, out_norm, out_flag) == B.OK
+        torch.cuda.synchronize()
+        assert float(out_norm.item()) == n * 2.0 ** -20 and int(out_flag.item()) == 0
+    # the oracle on the last ragged tile plus a sampled stretch agrees with the per-element value
+    lo = n - 5000
+    o_norm, o_flag = oracle.pg_norm2(start[lo:].cpu().numpy(), start[lo:].cpu().numpy(), p[lo:].cpu().numpy())
+    assert o_norm == 5000 * 2.0 ** -20 and o_flag == 0
+    p[n - 1] = float("nan")                                            # the very last element, in the last tile
+    assert static_norm(start, p, n, out_norm, out_flag) == B.OK
+    torch.cuda.synchronize()
+    assert int(out_flag.item()) == 1
+    del start, p
+    torch.cuda.empty_cache()
