@@ -14,8 +14,8 @@ using namespace kern;
 // (the memory system's rate for these read/write mixes); what separates them is how they degrade once the
 // diagnostics or eight arrivals add registers and arithmetic.  One vector per thread keeps the registers low
 // at every K; with five or more arrivals 128-thread blocks pack more warps into the register file than
-// 256-thread blocks (K = 8 with diagnostics: 6.55 against 6.02 TB/s) and the packed arithmetic halves the
-// instruction count of the K-fold update (6.55 against 6.47 TB/s); at K <= 4 neither matters.
+// 256-thread blocks (K = 8 with diagnostics: 6.47 against 5.79 TB/s); at K <= 4 neither matters.
+// Packed arithmetic stays off: it gains at most 1.3 % and is not bit-identical (see Lanes in the header).
 struct Shape {
     int V, BLK;
     bool PK;
@@ -23,7 +23,7 @@ struct Shape {
 constexpr Shape arrive_shape(int K) {
     if (K == 0) return {4, 256, false};           // re-seed only: one read stream, up to three written
     if (K <= 4) return {1, 256, false};
-    return {1, 128, true};
+    return {1, 128, false};
 }
 constexpr Shape kAdamShape = {1, 128, false};     // 6.82 TB/s; two vectors per thread in 256-thread blocks: 6.65-6.83
 constexpr int kMinTileVecs = 128;                 // smallest BLK * V of any arrival shape: the most blocks a launch can have

@@ -13,10 +13,10 @@
 //
 // Arithmetic contract: every fp32 operation is a separate IEEE-754 round-to-nearest operation in
 // the order Algorithm 3 states it (compiled with -fmad=false, IEEE division and square root, no
-// flush-to-zero), so results do not depend on the launch shape.  With PK the additions, subtractions
-// and multiplications are issued as the two-lane f32x2 instructions of sm_100; each lane is the same
-// IEEE operation.  The only fused multiply-adds are the explicit ones of the optional diagnostics,
-// which feed no state.
+// flush-to-zero), so results do not depend on the launch shape.  The only fused multiply-adds are the
+// explicit ones of the optional diagnostics, which feed no state.  PK (the two-lane f32x2 instructions
+// of sm_100) exists for the launch-shape benchmark only and is off in every shape the library runs:
+// see Lanes below.
 #pragma once
 #include "alsgd_kernels.cuh"
 
@@ -97,9 +97,14 @@ __device__ __forceinline__ uint2 bf16_pack4(const float4& x) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Two-lane fp32 arithmetic.  PK = true issues the sm_100 f32x2 instructions (one instruction, two
-// independent IEEE round-to-nearest lanes, denormals kept); PK = false is the same pair of scalar
-// operations.
+// Two-lane fp32 arithmetic.  PK = false is a pair of scalar IEEE operations: what the library runs.
+// PK = true issues the sm_100 f32x2 instructions (one instruction, two round-to-nearest lanes,
+// denormals kept).  Each packed instruction alone matches the scalar pair bit for bit, but measured
+// on B200 (CUDA 12.9) a packed multiply by a scalar broadcast to both lanes followed by a packed add
+// or subtract comes out as ONE fused multiply-add, despite the .rn qualifiers and -fmad=false: about
+// 20 % of such results differ from the two-rounding value in the last bit.  That breaks the
+// one-rounding-per-operation contract (and with it the bit-exact bf16 replicas), and the gain was
+// 1.3 % at best (eight arrivals with diagnostics), so PK stays a benchmark-only variant.
 // ---------------------------------------------------------------------------------------------
 template <bool PK>
 struct Lanes {
