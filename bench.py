@@ -550,7 +550,16 @@ def main_shape_sweep(args):
     torch.cuda.set_device(0)
     n = args.sweep_elems
     peak, which = measured_peak()
-    rows = sweep.run(n, reps=args.sweep_reps, warmup=3,
+    segments = None
+    if n == 109_549_056:             # the default size: AdamW walks the real weight-decay table of the 110M layout
+        from paper_2401_09135_b200 import binding as B, synth
+        tensors = synth.layout_110m()
+        P, offsets = B.alsgd_layout_size(tensors)
+        assert P == n
+        segments = sweep.decay_segments(tensors, offsets, P)
+    kinds = {"all": None, "adamw": sweep.KIND_ADAMW, "arrive": sweep.KIND_ARRIVE}[args.sweep_kind]
+    rows = sweep.run(n, reps=args.sweep_reps, warmup=3, segments=segments,
+                     select=(lambda v: v["kind"] == kinds) if kinds is not None else None,
                      log=(lambda r: print(json.dumps(r), file=sys.stderr, flush=True)) if args.verbose else None)
     best = {}
     for r in rows:
@@ -679,6 +688,7 @@ def main():
     ap.add_argument("--shape-sweep", action="store_true", help="time the launch shapes of libalsgd_sweep.so")
     ap.add_argument("--sweep-elems", type=int, default=109_549_056)
     ap.add_argument("--sweep-reps", type=int, default=10)
+    ap.add_argument("--sweep-kind", choices=["all", "adamw", "arrive"], default="all")
     ap.add_argument("--verbose", action="store_true")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

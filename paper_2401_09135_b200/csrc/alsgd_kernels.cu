@@ -25,7 +25,9 @@ constexpr Shape arrive_shape(int K) {
     if (K <= 4) return {1, 256, false};
     return {1, 128, false};
 }
-constexpr Shape kAdamShape = {1, 128, false};     // 6.82 TB/s; two vectors per thread in 256-thread blocks: 6.65-6.83
+// AdamW with the 110M layout's weight-decay table (every thread looks its segment up once, so one vector per
+// thread pays that latency twice as often): 2 x 128 6.79-6.82 TB/s, 2 x 64 6.79, 2 x 256 6.32-6.64, 1 x 128 6.47-6.51.
+constexpr Shape kAdamShape = {2, 128, false};
 constexpr int kMinTileVecs = 128;                 // smallest BLK * V of any arrival shape: the most blocks a launch can have
 
 template <int K, bool DIAG, int BASE, bool EXT>

@@ -72,7 +72,27 @@ def arrive_bytes_per_param(K, base_mode, phase):
 ADAMW_BYTES_PER_PARAM = 30
 
 
-def run(n, select=None, reps=10, warmup=3, phase_for=None, log=None):
+def decay_segments(tensors, offsets, P):
+    """Maximal runs of equal weight-decay flag over the flat vector (padding is its own undecayed run): the table
+    the AdamW kernel walks.  tensors have .numel and .decay."""
+    ends, flags = [], []
+
+    def push(end, flag):
+        if ends and flags[-1] == flag:
+            ends[-1] = end
+        else:
+            ends.append(end)
+            flags.append(flag)
+    for i, (t, off) in enumerate(zip(tensors, offsets)):
+        end = off + t.numel
+        push(end, 1 if t.decay else 0)
+        nxt = offsets[i + 1] if i + 1 < len(offsets) else P
+        if nxt != end:
+            push(nxt, 0)
+    return ends, flags
+
+
+def run(n, select=None, reps=10, warmup=3, phase_for=None, log=None, segments=None):
     """Time every variant (or those select(v) accepts) on vectors of n elements.  Returns a list of dicts with
     the variant's fields, the phase, ms per launch and GB/s on the algorithmic bytes."""
     import torch
@@ -95,9 +115,11 @@ def run(n, select=None, reps=10, warmup=3, phase_for=None, log=None):
     b.snapshot = hold(torch.empty(n, device=dev))
     b.adam_p, b.adam_m, b.adam_v = hold(f32(0.02)), hold(torch.zeros(n, device=dev)), hold(torch.zeros(n, device=dev))
     b.adam_g, b.adam_rep = hold(f32(0.01)), hold(torch.empty(n, device=dev, dtype=torch.int16))
-    b.seg_end = hold(torch.tensor([n], device=dev, dtype=torch.int64))
-    b.seg_decay = hold(torch.tensor([1], device=dev, dtype=torch.int32))
-    b.n_seg = 1
+    seg_end, seg_decay = segments if segments is not None else ([n], [1])
+    assert seg_end[-1] == n
+    b.seg_end = hold(torch.tensor(seg_end, device=dev, dtype=torch.int64))
+    b.seg_decay = hold(torch.tensor(seg_decay, device=dev, dtype=torch.int32))
+    b.n_seg = len(seg_end)
     b.diag_scratch = hold(torch.zeros(8 * (n // 256 + 66), device=dev, dtype=torch.float64))
     b.diag_out = hold(torch.zeros(8, device=dev, dtype=torch.float64))
     b.diag_flags = hold(torch.zeros(8, device=dev, dtype=torch.int32))
