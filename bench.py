@@ -44,16 +44,17 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter from the committed ncu captures
 # (profiles/), valid only for the kernel source they were taken from.
 NCU_TRAFFIC = {
-    "src_sha256": "096949379a0ffd9f559f91c7bc7f061aede597ccb5d156faabf1363cc667106a",
-    "adamw_bytes_per_param": 28.90,     # ncu capture at P = 50.3M elements, scaled by P
+    "src_sha256": "d54a53f8760243240cdc90273f6e6eebb2c920e34f9114079b8638d4a4f1122e",
+    "adamw_bytes_per_param": 28.91,     # ncu capture at P = 50.3M elements (profiles/adamw_kernel_flat48M.md), scaled by P
     "arrive_bytes_per_param": 28.90,    # same capture, K = 1, average over one Delayed-Nesterov cycle
 }
 
 
 def kernel_source_hash():
     h = hashlib.sha256()
-    with open(os.path.join(ROOT, "paper_2401_09135_b200", "csrc", "alsgd_kernels.cu"), "rb") as f:
-        h.update(f.read())
+    for name in ("alsgd_kernels_impl.cuh", "alsgd_kernels.cu"):
+        with open(os.path.join(ROOT, "paper_2401_09135_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
     return h.hexdigest()
 
 

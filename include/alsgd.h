@@ -334,6 +334,19 @@ int alsgd_sched_next_batch(alsgd_sched* s, uint32_t* ids_out, double* times_out,
 /* Total local updates synchronised so far (Algorithm 2's t_local). */
 int alsgd_sched_local_updates(alsgd_sched* s, uint64_t* t_local_out);
 
+/* Checkpoint / resume of the scheduler, the counterpart of alsgd_export_state for Algorithm 2's own state:
+ * tau_grace, t_max, t_local and per worker the job in flight (completion time, local updates), whether it ever
+ * ran and the restart time its last window gave it (tau_sync + tau_grace).  An image imported into a scheduler
+ * created for the same number of workers continues the timeline exactly where it stopped: the same windows, ids,
+ * times and restart times.  All host memory; a few dozen bytes per worker.
+ *   alsgd_sched_state_bytes   size of the image
+ *   alsgd_sched_export        host_dst: `bytes` >= that size (ALSGD_E_NOMEM otherwise)
+ *   alsgd_sched_import        ALSGD_E_ARG: not a scheduler image, another worker count, or fields outside their
+ *                             domain; the scheduler is unchanged then */
+int alsgd_sched_state_bytes(alsgd_sched* s, uint64_t* bytes_out);
+int alsgd_sched_export(alsgd_sched* s, void* host_dst, uint64_t bytes);
+int alsgd_sched_import(alsgd_sched* s, const void* host_src, uint64_t bytes);
+
 /* ------------------------------------------------------------------------------------------------
  * Diagnostics without any allocation (the paper has no counterpart; this serves embedders)
  * ---------------------------------------------------------------------------------------------- */

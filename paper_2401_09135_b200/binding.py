@@ -95,6 +95,9 @@ SIGNATURES = {
     "alsgd_sched_dispatch": (C.c_int, [_vp, C.c_uint32, C.c_double, C.c_uint32]),
     "alsgd_sched_next_batch": (C.c_int, [_vp, _u32p, _f64p, C.c_uint32, _u32p, _f64p]),
     "alsgd_sched_local_updates": (C.c_int, [_vp, _u64p]),
+    "alsgd_sched_state_bytes": (C.c_int, [_vp, _u64p]),
+    "alsgd_sched_export": (C.c_int, [_vp, _vp, C.c_uint64]),
+    "alsgd_sched_import": (C.c_int, [_vp, _vp, C.c_uint64]),
     "alsgd_pg_norm_static": (C.c_int, [_vp, _vp, C.c_uint64, C.c_int32, _vp, _vp, _vp]),
 }
 STATIC_MAX_ELEMS = 1 << 27
@@ -213,6 +216,16 @@ class Scheduler:
         out = C.c_uint64()
         _check(lib().alsgd_sched_local_updates(self._h, C.byref(out)), "alsgd_sched_local_updates")
         return int(out.value)
+
+    def export_state(self) -> bytes:
+        n = C.c_uint64()
+        _check(lib().alsgd_sched_state_bytes(self._h, C.byref(n)), "alsgd_sched_state_bytes")
+        buf = C.create_string_buffer(int(n.value))
+        _check(lib().alsgd_sched_export(self._h, buf, int(n.value)), "alsgd_sched_export")
+        return buf.raw
+
+    def import_state(self, image: bytes):
+        _check(lib().alsgd_sched_import(self._h, image, len(image)), "alsgd_sched_import")
 
     def close(self):
         if self._h:

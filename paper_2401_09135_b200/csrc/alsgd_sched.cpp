@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstring>
 #include <new>
 #include <vector>
 
@@ -146,6 +147,76 @@ int alsgd_sched_next_batch(alsgd_sched* s, uint32_t* ids_out, double* times_out,
     s->t_local = t_local;
     *k_out = k;
     if (restart_out) *restart_out = restart;
+    return ALSGD_OK;
+}
+
+namespace {
+
+// Image of a scheduler: header, then one record per worker.  Plain fixed-width fields, host byte order.
+struct SchedImageHeader {
+    char magic[8];
+    uint32_t version;
+    uint32_t n_workers;
+    double tau_grace;
+    uint64_t t_max;
+    uint64_t t_local;
+};
+struct SchedImageJob {
+    double completed_time;
+    double restart_time;
+    uint32_t local_updates;
+    uint8_t in_flight;
+    uint8_t ran_before;
+    uint8_t reserved[2];
+};
+const char kSchedMagic[8] = {'A', 'L', 'S', 'G', 'D', 'S', 'C', '1'};
+
+}  // namespace
+
+int alsgd_sched_state_bytes(alsgd_sched* s, uint64_t* bytes_out) {
+    if (!s || !bytes_out) return ALSGD_E_ARG;
+    *bytes_out = sizeof(SchedImageHeader) + sizeof(SchedImageJob) * (uint64_t)s->n;
+    return ALSGD_OK;
+}
+
+int alsgd_sched_export(alsgd_sched* s, void* host_dst, uint64_t bytes) {
+    if (!s || !host_dst) return ALSGD_E_ARG;
+    if (bytes < sizeof(SchedImageHeader) + sizeof(SchedImageJob) * (uint64_t)s->n) return ALSGD_E_NOMEM;
+    SchedImageHeader h{};
+    std::memcpy(h.magic, kSchedMagic, 8);
+    h.version = 1; h.n_workers = s->n; h.tau_grace = s->tau_grace; h.t_max = s->t_max; h.t_local = s->t_local;
+    uint8_t* out = static_cast<uint8_t*>(host_dst);
+    std::memcpy(out, &h, sizeof(h));
+    out += sizeof(h);
+    for (const Job& j : s->jobs) {
+        SchedImageJob r{};
+        r.completed_time = j.completed_time; r.restart_time = j.restart_time; r.local_updates = j.local_updates;
+        r.in_flight = j.in_flight ? 1 : 0; r.ran_before = j.ran_before ? 1 : 0;
+        std::memcpy(out, &r, sizeof(r));
+        out += sizeof(r);
+    }
+    return ALSGD_OK;
+}
+
+int alsgd_sched_import(alsgd_sched* s, const void* host_src, uint64_t bytes) {
+    if (!s || !host_src || bytes < sizeof(SchedImageHeader)) return ALSGD_E_ARG;
+    const uint8_t* in = static_cast<const uint8_t*>(host_src);
+    SchedImageHeader h;
+    std::memcpy(&h, in, sizeof(h));
+    if (std::memcmp(h.magic, kSchedMagic, 8) != 0 || h.version != 1 || h.n_workers != s->n) return ALSGD_E_ARG;
+    if (bytes < sizeof(SchedImageHeader) + sizeof(SchedImageJob) * (uint64_t)s->n) return ALSGD_E_ARG;
+    if (!(h.tau_grace >= 0.0) || !std::isfinite(h.tau_grace)) return ALSGD_E_ARG;
+    in += sizeof(h);
+    std::vector<Job> jobs(s->n);
+    for (uint32_t w = 0; w < s->n; ++w) {
+        SchedImageJob r;
+        std::memcpy(&r, in + sizeof(r) * (uint64_t)w, sizeof(r));
+        if (r.in_flight > 1 || r.ran_before > 1 || !std::isfinite(r.completed_time) || !std::isfinite(r.restart_time)) return ALSGD_E_ARG;
+        jobs[w].completed_time = r.completed_time; jobs[w].restart_time = r.restart_time;
+        jobs[w].local_updates = r.local_updates; jobs[w].in_flight = r.in_flight != 0; jobs[w].ran_before = r.ran_before != 0;
+    }
+    s->jobs.swap(jobs);
+    s->tau_grace = h.tau_grace; s->t_max = h.t_max; s->t_local = h.t_local;
     return ALSGD_OK;
 }
 

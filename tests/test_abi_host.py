@@ -287,3 +287,53 @@ def test_benchmark_reference_arm_needs_only_the_oracle():
     import bench
     lib_steps, lib_order = bench.build_schedule(40)
     assert steps == lib_steps == [16, 25, 33, 50] and order == lib_order
+
+
+def test_scheduler_checkpoint_continues_the_timeline():
+    """Algorithm 2 for 20 windows; export after 9; a fresh scheduler that imports the image produces the
+    identical remaining windows (ids, times, restart time, t_local)."""
+    W, speeds = 5, [1.0, 1.3, 1.7, 2.2, 3.0]
+    steps = B.alsgd_dylu_steps(speeds, 40)
+    dur = synth.job_durations(speeds, steps, 64, synth.SEED + 21)
+
+    def drive(s, rounds, n_windows, log):
+        for _ in range(n_windows):
+            ids, times, restart = s.next_batch()
+            log.append((ids, times, restart, s.local_updates()))
+            for w in ids:
+                rounds[w] += 1
+                s.dispatch(w, dur[w, rounds[w]], steps[w])
+
+    full, rounds = [], [0] * W
+    a = B.Scheduler(W, 0.35)
+    for w in range(W):
+        a.dispatch(w, dur[w, 0], steps[w])
+    drive(a, rounds, 9, full)
+    image = a.export_state()
+    rounds_at_9 = list(rounds)
+    drive(a, rounds, 11, full)
+    assert any(len(ids) > 1 for ids, *_ in full) and any(len(ids) == 1 for ids, *_ in full)
+
+    b = B.Scheduler(W, 0.0)                      # other grace period: the image brings its own
+    b.import_state(image)
+    resumed = []
+    drive(b, rounds_at_9, 11, resumed)
+    assert resumed == full[9:]
+
+    L = B.lib()
+    c = B.Scheduler(W + 1, 0.35)
+    assert L.alsgd_sched_import(c._h, image, len(image)) == B.E_ARG            # other worker count
+    assert L.alsgd_sched_import(b._h, image[:20], 20) == B.E_ARG               # truncated
+    assert L.alsgd_sched_import(b._h, b"x" * len(image), len(image)) == B.E_ARG
+    small = C.create_string_buffer(8)
+    assert L.alsgd_sched_export(b._h, small, 8) == B.E_NOMEM
+    # a mid-window export: one job consumed, others in flight
+    d = B.Scheduler(2, 10.0)
+    d.dispatch(0, 1.0, 3)
+    img0 = d.export_state()
+    d.dispatch(1, 2.0, 4)
+    e = B.Scheduler(2, 0.0)
+    e.import_state(img0)
+    assert L.alsgd_sched_dispatch(e._h, 0, 1.0, 3) == B.E_STATE                # worker 0's job is in flight in the image
+    e.dispatch(1, 2.0, 4)
+    assert e.next_batch() == d.next_batch()
