@@ -422,6 +422,8 @@ def run_ksweep(args, device=0):
     torch.cuda.set_device(device)
     tensors = synth.layout_110m()
     W, N, inner = 8, 8, 10
+    diag = bool(getattr(args, "diag", False))
+    arrive_flags = B.ARRIVE_RESEED | ((B.ARRIVE_NORM | B.ARRIVE_NANCHECK) if diag else 0)
     peak, which = measured_peak()
     out = []
     gpool = None
@@ -441,7 +443,7 @@ def run_ksweep(args, device=0):
             e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
             e0.record()
             for i in range(0, W, k):
-                ctx.alsgd_arrive(order[i:i + k], B.ARRIVE_RESEED, want_info=False)
+                ctx.alsgd_arrive(order[i:i + k], arrive_flags, want_info=False)
             e1.record()
             for w in range(W):
                 for _ in range(inner):
@@ -471,7 +473,8 @@ def run_ksweep(args, device=0):
         ctx.close()
         del ctx
         torch.cuda.empty_cache()
-    return {"workload": "decoder-110M W=8 N=8 beta=0.9 outer_lr=0.7, k-sweep, 10 inner AdamW steps per worker per round",
+    return {"workload": "decoder-110M W=8 N=8 beta=0.9 outer_lr=0.7, k-sweep, 10 inner AdamW steps per worker per round"
+                        + (", squared-norm and non-finite diagnostics on every arrival" if diag else ""),
             "peak_gbs": peak, "peak_source": f"of {which}", "unit": "GB/s", "rounds_timed": len(ev), "sweep": out}
 
 
@@ -683,6 +686,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the k-sweep and layout tables of the default line")
     ap.add_argument("--ksweep", action="store_true", help="arrival-batch sweep (k = 1, 2, 4, 8) with 8 resident workers")
+    ap.add_argument("--diag", action="store_true", help="with --ksweep: request the diagnostics on every arrival")
     ap.add_argument("--layouts", action="store_true", help="per-kernel throughput on 23M / 60M / 110M / 150M layouts")
     ap.add_argument("--cpu-kernels", action="store_true", help="time the oracle's loops per kernel on the host cores")
     ap.add_argument("--profile-case", choices=["single", "batches", "diag"], help="run a small fixed case for a profiler capture")

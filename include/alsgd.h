@@ -166,7 +166,8 @@ int alsgd_inner_adamw_bf16(alsgd_ctx* ctx, uint32_t worker, const uint16_t* grad
 typedef struct alsgd_arrival_info {
     uint64_t tick;       /* Algorithm 3's t at which this arrival was applied */
     uint64_t staleness;  /* tick minus the worker's pull tick */
-    double gnorm2;       /* sum of squared pseudo-gradient entries (0 unless NORM) */
+    double gnorm2;       /* sum of squared pseudo-gradient entries (0 unless NORM); squares are formed in binary32, so an
+                            entry beyond 1.8e19 in magnitude makes it +inf although the entry is finite */
     uint32_t worker;
     uint32_t boundary;   /* 1 if (t+1) % N == 0: momentum updated, buffer reset */
     uint32_t nonfinite;  /* 1 if any entry was NaN or Inf (0 unless NANCHECK) */

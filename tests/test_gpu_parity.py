@@ -492,3 +492,44 @@ def test_nonfinite_worker_is_flagged_not_trapped():
     assert [i["nonfinite"] for i in info] == [0, 1]
     pair.check_all("after poisoned arrival")       # NaN/Inf propagate exactly as the definition says
     pair.close()
+
+
+@pytest.mark.parametrize("pg_current,buffered,N", [(False, False, 4), (True, False, 3), (False, True, 16), (True, True, 2)])
+def test_nonfinite_flags_per_arrival_in_every_mode(pg_current, buffered, N):
+    """The per-arrival non-finite flag comes from a replay that only runs where the state left by the batch is
+    not finite.  Poisoned entries in a vector body, in the scalar tail and in several arrivals of one batch; an
+    overflow that is not a non-finite entry; batches that follow on an already poisoned model; batches of eight
+    that share one dispatch snapshot."""
+    P = 4 * 4099 + 3                                   # scalar tail of three elements
+    W = 8
+    pair = Pair(synth.flat_tensors(P), W, N, 0.9, 0.7, align=1, pg_current=pg_current, buffered=buffered)
+    start(pair, SEED + 17)
+    r = np.random.default_rng(17)
+
+    def round_of(ids, poison):
+        for w in ids:
+            z = synth.normal_vec(P, 1e-3, SEED + 17, synth.STREAM_DELTA, sub=int(r.integers(0, 1 << 20)))
+            for where, value in poison.get(w, []):
+                z[where] = value
+            pair.perturb(w, dev(z), z)
+        with np.errstate(all="ignore"):
+            info = pair.arrive(ids, reseed=True, norm=True)      # flags and norms are compared with the oracle inside
+            pair.check_all(f"batch {ids}")
+        return [i["nonfinite"] for i in info]
+
+    assert round_of([0, 1, 2, 3, 4, 5, 6, 7], {}) == [0] * 8                        # clean, distinct snapshots
+    assert round_of([3, 1, 4, 0, 5, 2, 7, 6], {}) == [0] * 8                        # clean, one shared snapshot
+    # a finite entry large enough to overflow theta and the sum of squares: not a non-finite entry
+    flags = round_of([2, 6], {6: [(11, np.float32(-3e38))]})
+    assert flags == ([0, 0] if not pg_current else flags) and flags[0] == 0
+    # Inf in a vector body of one arrival, NaN in the scalar tail of another, both in one batch of eight
+    flags = round_of([7, 0, 1, 2, 3, 4, 5, 6], {1: [(4000, np.inf)], 4: [(P - 1, np.nan)]})
+    if not pg_current:
+        assert flags == [0, 0, 1, 0, 0, 1, 0, 0]
+    else:                                             # later arrivals see the poisoned running theta
+        assert flags[:2] == [0, 0] and flags[2] == 1 and flags[5] == 1
+    # the model is poisoned now; against the dispatch snapshot (also poisoned at those elements) or the running theta
+    # the oracle decides, element by element, what each arrival's pseudo-gradient holds
+    round_of([0, 1], {})
+    round_of([5], {5: [(123, -np.inf)]})
+    pair.close()
