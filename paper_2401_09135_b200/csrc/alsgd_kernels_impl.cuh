@@ -160,11 +160,11 @@ __device__ __forceinline__ bool nonfinite_bits(float x) { return (__float_as_uin
 // DIAG accumulates the squares of the (unmodified) pseudo-gradient entries into acc.
 template <bool PK, bool DIAG, int BASE, bool EXT>
 __device__ __forceinline__ void dn_step(float2& th, float2& d, float2& mm, float2 b, float2 p, bool boundary, float w,
-                                        const ArriveArgs& a, float2& acc) {
+                                        const ArriveArgs& a, float& acc) {
     using L = Lanes<PK>;
     const float2 start = (BASE == kBaseCurrent) ? th : b;
     float2 g = L::sub(start, p);                              // pseudo-gradient
-    if (DIAG) acc = L::fma(g, g, acc);                        // sum of squares (at most 8 terms per lane in fp32)
+    if (DIAG) acc = __fmaf_rn(g.y, g.y, __fmaf_rn(g.x, g.x, acc));   // sum of squares (at most 16 terms per thread in fp32)
     if (EXT) {
         if (a.flags & kDelayComp) {                           // g + lambda * g*g*(theta_now - theta_at_dispatch)
             const float2 drift = L::sub(th, start);
@@ -208,7 +208,7 @@ __device__ __noinline__ uint32_t replay_nonfinite(const ArriveArgs& a, uint64_t 
     float2 th = make_float2(ld1(gd, a.theta + e, kGuardTheta), 0.f);
     float2 d = make_float2((a.flags & kDeltaZeroIn) ? 0.f : ld1(gd, a.delta + e, kGuardDelta), 0.f);
     float2 mm = make_float2((a.flags & kReadM) ? ld1(gd, a.mom + e, kGuardMom) : 0.f, 0.f);
-    float2 unused = make_float2(0.f, 0.f);
+    float unused = 0.f;
 #pragma unroll 1
     for (int j = 0; j < K; ++j) {
         const float p = ld1(gd, a.p[j] + e, kGuardWorkerP);
@@ -219,6 +219,31 @@ __device__ __noinline__ uint32_t replay_nonfinite(const ArriveArgs& a, uint64_t 
                                              (a.boundary_mask >> j) & 1u, EXT ? a.w[j] : 1.0f, a, unused);
     }
     return bad;
+}
+
+// Sum over the 32 lanes of a warp of K values per lane with K - 1 + (5 - log2 K') shuffles instead of 5 K
+// (K' = K rounded up to a power of two): in each of the first log2 K' steps a lane hands half of its values to
+// its partner and adds the partner's other half to the half it keeps; afterwards every lane holds one value, and
+// the remaining steps are ordinary.  On return lane l with (l & (32 / K' - 1)) == 0 holds the warp's sum of value
+// j = l / (32 / K').  The order of the additions is fixed, so the result is reproducible.
+template <int K>
+__device__ __forceinline__ float warp_sum_transposed(float (&v)[8], int lane) {
+    constexpr int KP = K <= 1 ? 1 : K <= 2 ? 2 : K <= 4 ? 4 : 8;
+    int m = 16;
+#pragma unroll
+    for (int cnt = KP; cnt > 1; cnt >>= 1, m >>= 1) {
+        const bool upper = lane & m;
+#pragma unroll
+        for (int i = 0; i < cnt / 2; ++i) {
+            const float send = upper ? v[i] : v[i + cnt / 2];
+            const float keep = upper ? v[i + cnt / 2] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, m);
+        }
+    }
+    float s = v[0];
+#pragma unroll
+    for (; m > 0; m >>= 1) s = s + __shfl_xor_sync(0xFFFFFFFFu, s, m);
+    return s;
 }
 
 template <int K, int V, int BLK, int MINB, bool DIAG, int BASE, bool EXT, bool PERSIST, bool PK>
@@ -236,9 +261,9 @@ __global__ void __launch_bounds__(BLK, MINB) arrive_kernel(const __grid_constant
     const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
     const DebugGuard& gd = a.guard;
 
-    float2 acc[KK];                                            // per arrival: sums of squares, two lanes
+    float acc[KK];                                             // per arrival: sum of squares of this thread's entries
 #pragma unroll
-    for (int j = 0; j < KK; ++j) acc[j] = make_float2(0.f, 0.f);
+    for (int j = 0; j < KK; ++j) acc[j] = 0.f;
     uint32_t bad = 0;                                          // bit j: arrival j had a non-finite entry
 
     float4* __restrict__ theta4 = reinterpret_cast<float4*>(a.theta);
@@ -359,13 +384,12 @@ __global__ void __launch_bounds__(BLK, MINB) arrive_kernel(const __grid_constant
     if (DIAG && K > 0) {
         __shared__ float warp_sum[BLK / 32][KK];
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        constexpr int KP = K <= 1 ? 1 : K <= 2 ? 2 : K <= 4 ? 4 : 8;
+        float v[8];
 #pragma unroll
-        for (int j = 0; j < K; ++j) {
-            float s = acc[j].x + acc[j].y;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s = s + __shfl_down_sync(0xFFFFFFFFu, s, o);
-            if (lane == 0) warp_sum[warp][j] = s;
-        }
+        for (int j = 0; j < 8; ++j) v[j] = j < K ? acc[j < K ? j : 0] : 0.f;
+        const float s = warp_sum_transposed<K>(v, lane);
+        if ((lane & (32 / KP - 1)) == 0 && lane / (32 / KP) < K) warp_sum[warp][lane / (32 / KP)] = s;
         bad = __reduce_or_sync(0xFFFFFFFFu, bad);
         if (lane == 0 && bad) {
             for (int j = 0; j < K; ++j)

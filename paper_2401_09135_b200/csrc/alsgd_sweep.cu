@@ -94,10 +94,10 @@ cudaError_t run_adamw(const alsgd_sweep_buffers& b, uint32_t, cudaStream_t s) {
     ARR(K, 4, 128, 1, DIAG, BASE, 0, 0) ARR(K, 4, 128, 1, DIAG, BASE, 0, 1) \
     ARR(K, 4, 256, 1, DIAG, BASE, 0, 0) ARR(K, 4, 256, 1, DIAG, BASE, 0, 1)
 #define ARR_DIAG_SHAPES(K, BASE)                                      \
+    ARR(K, 1, 64, 1, 1, BASE, 0, 0)                                   \
     ARR(K, 1, 128, 1, 1, BASE, 0, 0) ARR(K, 1, 128, 1, 1, BASE, 0, 1) \
     ARR(K, 1, 256, 1, 1, BASE, 0, 0) ARR(K, 1, 256, 1, 1, BASE, 0, 1) \
-    ARR(K, 2, 128, 1, 1, BASE, 0, 0) ARR(K, 2, 128, 1, 1, BASE, 0, 1) \
-    ARR(K, 2, 256, 1, 1, BASE, 0, 0) ARR(K, 2, 256, 1, 1, BASE, 0, 1)
+    ARR(K, 2, 128, 1, 1, BASE, 0, 0) ARR(K, 2, 256, 1, 1, BASE, 0, 0)
 
 const Entry kEntries[] = {
     ADM(1, 64, 1, 0) ADM(1, 128, 1, 0) ADM(1, 256, 1, 0) ADM(1, 512, 1, 0) ADM(1, 1024, 1, 0)
@@ -119,6 +119,8 @@ const Entry kEntries[] = {
     ARR(8, 1, 256, 4, 0, kBaseShared, 0, 0) ARR(8, 1, 128, 8, 0, kBaseShared, 0, 0)
     ARR(4, 2, 256, 3, 0, kBasePerArrival, 0, 0) ARR(4, 2, 256, 3, 0, kBaseShared, 0, 0)
     ARR(1, 4, 256, 3, 0, kBasePerArrival, 0, 0) ARR(1, 4, 128, 6, 0, kBasePerArrival, 0, 0)
+    ARR(8, 1, 128, 6, 1, kBaseShared, 0, 0) ARR(8, 1, 128, 7, 1, kBaseShared, 0, 0)
+    ARR(8, 1, 128, 5, 1, kBasePerArrival, 0, 0) ARR(8, 1, 64, 12, 1, kBaseShared, 0, 0)
 };
 constexpr int kCount = (int)(sizeof(kEntries) / sizeof(kEntries[0]));
 
