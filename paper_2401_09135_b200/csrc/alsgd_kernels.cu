@@ -13,8 +13,9 @@ using namespace kern;
 // every one-tile-per-block shape with at most ~20 vectors in flight per thread lands within 1 % of 6.8 TB/s
 // (the memory system's rate for these read/write mixes); what separates them is how they degrade once the
 // diagnostics or eight arrivals add registers and arithmetic.  One vector per thread keeps the registers low
-// at every K; with five or more arrivals 128-thread blocks pack more warps into the register file than
-// 256-thread blocks (K = 8 with diagnostics: 6.47 against 5.79 TB/s); at K <= 4 neither matters.
+// at every K (K = 8: 69-96 registers; two vectors per thread lose 2-10 %, four up to 40 %); with five or more
+// arrivals 128-thread blocks fit more warps into the register file than 256-thread blocks (96 registers: five
+// blocks of four warps against two of eight), worth about 0.5 %; at K <= 4 neither matters.
 // Packed arithmetic stays off: it gains at most 1.3 % and is not bit-identical (see Lanes in the header).
 struct Shape {
     int V, BLK;
