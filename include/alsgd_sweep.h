@@ -30,7 +30,9 @@ typedef struct alsgd_sweep_variant {
     uint32_t persistent; /* 1: grid of resident blocks looping over tiles; 0: one tile per block */
     uint32_t packed;     /* 1: f32x2 two-lane arithmetic */
     uint32_t diag;       /* 1: with the squared-norm / non-finite diagnostics */
-    uint32_t reserved;
+    uint32_t staged;     /* 0: operands move through registers (128-bit loads and stores); otherwise the tile size in
+                            elements of a variant that moves every stream with 1-D bulk copies (cp.async.bulk global ->
+                            shared with an mbarrier, arithmetic from shared memory, cp.async.bulk shared -> global) */
 } alsgd_sweep_variant;
 
 /* All pointers are device pointers to caller-owned buffers of n elements (16-byte aligned), except where noted. */
@@ -64,7 +66,9 @@ typedef struct alsgd_sweep_buffers {
 int alsgd_sweep_count(void);
 /* idx in [0, count).  Returns 0, or -1 for a bad index or null pointer. */
 int alsgd_sweep_describe(int idx, alsgd_sweep_variant* out);
-/* Enqueue one launch of variant idx on the stream (cudaStream_t).  Returns 0 or the cudaError_t of the launch. */
+/* Enqueue one launch of variant idx on the stream (cudaStream_t).  Returns 0 or the cudaError_t of the launch.
+ * Staged variants need n to be a multiple of 8 and 16-byte aligned buffers (cudaErrorInvalidValue otherwise) and
+ * record a wait that ran out in b->diag_flags[7] instead of hanging. */
 int alsgd_sweep_launch(int idx, const alsgd_sweep_buffers* b, uint32_t phase, void* stream);
 
 #ifdef __cplusplus

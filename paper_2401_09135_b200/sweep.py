@@ -19,7 +19,7 @@ BASE_NAMES = {0: "per-arrival", 1: "shared", 2: "current"}
 
 class Variant(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("kind", "K", "base_mode", "V", "block", "min_blocks", "persistent",
-                                          "packed", "diag", "reserved")]
+                                          "packed", "diag", "staged")]
 
 
 class Buffers(C.Structure):
@@ -56,7 +56,7 @@ def variants():
     for i in range(L.alsgd_sweep_count()):
         v = Variant()
         assert L.alsgd_sweep_describe(i, C.byref(v)) == 0
-        out.append({n: int(getattr(v, n)) for n, _ in Variant._fields_ if n != "reserved"})
+        out.append({n: int(getattr(v, n)) for n, _ in Variant._fields_})
         out[-1]["index"] = i
     return out
 
@@ -122,7 +122,8 @@ def run(n, select=None, reps=10, warmup=3, phase_for=None, log=None, segments=No
     b.n_seg = len(seg_end)
     b.diag_scratch = hold(torch.zeros(8 * (n // 256 + 66), device=dev, dtype=torch.float64))
     b.diag_out = hold(torch.zeros(8, device=dev, dtype=torch.float64))
-    b.diag_flags = hold(torch.zeros(8, device=dev, dtype=torch.int32))
+    keep_flags = torch.zeros(8, device=dev, dtype=torch.int32)
+    b.diag_flags = hold(keep_flags)
     stream = torch.cuda.current_stream().cuda_stream
     rows = []
     for v in variants():
@@ -144,6 +145,8 @@ def run(n, select=None, reps=10, warmup=3, phase_for=None, log=None, segments=No
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / reps
+        if v["staged"] and int(keep_flags[7].item()) != 0:
+            raise RuntimeError(f"sweep variant {v}: a bounded wait ran out")
         row = dict(v, phase=phase, bytes_per_param=bpp, ms=ms, gbs=bpp * n / ms / 1e6)
         rows.append(row)
         if log:
