@@ -63,6 +63,10 @@ typedef struct alsgd_sweep_buffers {
 #define ALSGD_SWEEP_PHASE_MIDDLE 0u  /* Delta read and written, no momentum boundary in the batch */
 #define ALSGD_SWEEP_PHASE_CYCLE 1u   /* the batch is a whole cycle (N = K): Delta neither read nor written, m read and written */
 
+/* OR-ed into `phase`: launch as a programmatic dependent launch (the kernel's blocks may be placed while the previous
+ * kernel of the stream drains and wait, before their first memory access, for its completion).  Register variants only. */
+#define ALSGD_SWEEP_LAUNCH_DEPENDENT 0x100u
+
 int alsgd_sweep_count(void);
 /* idx in [0, count).  Returns 0, or -1 for a bad index or null pointer. */
 int alsgd_sweep_describe(int idx, alsgd_sweep_variant* out);

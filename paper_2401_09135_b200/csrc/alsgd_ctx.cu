@@ -463,7 +463,7 @@ int adamw_impl(alsgd_ctx* c, uint32_t worker, const void* grads, bool bf16, int 
         a.g16 = bf16 ? static_cast<const uint16_t*>(gsrc) : nullptr;
         a.n = len;
         a.seg_base = lo;
-        return launch_adamw(a, c->stream);
+        return launch_adamw(a, grads_is_device != 0, c->stream);
     };
     if (grads_is_device) {
         ALSGD_CUDA(c, launch_range(0, c->P, grads));

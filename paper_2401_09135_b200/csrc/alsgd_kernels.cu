@@ -39,7 +39,10 @@ cudaError_t launch_arrive_k(const ArriveArgs& a, cudaStream_t s) {
     unsigned grid = 1;
     cudaError_t e = grid_for(a.n, (uint64_t)sh.V * sh.BLK, &grid);
     if (e != cudaSuccess) return e;
-    kern<<<grid, sh.BLK, 0, s>>>(a);
+    // Programmatic dependent launch: the blocks may be placed while the stream's previous kernel drains (they wait
+    // for its completion before their first access); at 23M elements this hides 1-2 % of launch gap, at 110M ~0.
+    e = launch_kernel(kern, grid, sh.BLK, s, a, true);
+    if (e != cudaSuccess) return e;
     if (DIAG && K > 0) {
         double* chunk_sum = a.diag_partial + (uint64_t)K * grid;        // behind the K x grid partials
         diag_reduce1_kernel<<<dim3(kDiagChunks, K), kDiagBlock, 0, s>>>(a.diag_partial, grid, chunk_sum);
@@ -89,15 +92,14 @@ cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics
     return launch_arrive_d<kBasePerArrival>(a, diagnostics, extended, s);
 }
 
-cudaError_t launch_adamw(const AdamArgs& a, cudaStream_t s) {
+cudaError_t launch_adamw(const AdamArgs& a, bool dependent_launch, cudaStream_t s) {
     if (a.n == 0) return cudaSuccess;
     constexpr Shape sh = kAdamShape;
     unsigned grid = 1;
     cudaError_t e = grid_for(a.n, (uint64_t)sh.V * sh.BLK, &grid);
     if (e != cudaSuccess) return e;
-    if (a.g16) adamw_kernel<sh.V, sh.BLK, 1, true, false><<<grid, sh.BLK, 0, s>>>(a);
-    else adamw_kernel<sh.V, sh.BLK, 1, false, false><<<grid, sh.BLK, 0, s>>>(a);
-    return cudaGetLastError();
+    if (a.g16) return launch_kernel(adamw_kernel<sh.V, sh.BLK, 1, true, false>, grid, sh.BLK, s, a, dependent_launch);
+    return launch_kernel(adamw_kernel<sh.V, sh.BLK, 1, false, false>, grid, sh.BLK, s, a, dependent_launch);
 }
 
 }  // namespace alsgd

@@ -79,6 +79,8 @@ struct AdamArgs {
 uint64_t diag_partial_count(uint64_t n);
 
 cudaError_t launch_arrive(const ArriveArgs& a, bool pg_current, bool diagnostics, bool extended, cudaStream_t s);
-cudaError_t launch_adamw(const AdamArgs& a, cudaStream_t s);
+// dependent_launch: allow the kernel's blocks to be placed while the stream's previous kernel drains (off where
+// the launch also waits on an event of another stream).
+cudaError_t launch_adamw(const AdamArgs& a, bool dependent_launch, cudaStream_t s);
 
 }  // namespace alsgd

@@ -246,8 +246,34 @@ __device__ __forceinline__ float warp_sum_transposed(float (&v)[8], int lane) {
     return s;
 }
 
+// Programmatic dependent launch: when a kernel is launched with the stream-serialization attribute its blocks
+// may be placed on the SMs while the previous kernel of the stream is still draining; they then wait here, before
+// their first memory access, until that kernel has completed and its writes are visible.  launch_dependents lets
+// the next kernel do the same with this one.  Without the attribute both instructions do nothing.
+__device__ __forceinline__ void grid_dependency_sync() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+// kernel<<<grid, block, 0, s>>>(args), optionally as a programmatic dependent launch.
+template <typename Args>
+inline cudaError_t launch_kernel(void (*kern)(Args), unsigned grid, unsigned block, cudaStream_t s, const Args& args, bool pdl) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, args);
+}
+
 template <int K, int V, int BLK, int MINB, bool DIAG, int BASE, bool EXT, bool PERSIST, bool PK>
 __global__ void __launch_bounds__(BLK, MINB) arrive_kernel(const __grid_constant__ ArriveArgs a) {
+    grid_dependency_sync();
     constexpr int KK = K > 0 ? K : 1;
     constexpr int NB = (BASE == kBasePerArrival) ? KK : 1;     // snapshot vectors held in registers
     const uint64_t nvec = a.n >> 2;
@@ -486,6 +512,7 @@ __device__ __forceinline__ float4 widen_bf16x4(uint2 b) {
 
 template <int V, int BLK, int MINB, bool G16, bool PERSIST>
 __global__ void __launch_bounds__(BLK, MINB) adamw_kernel(const __grid_constant__ AdamArgs a) {
+    grid_dependency_sync();
     const uint64_t nvec = a.n >> 2;
     const uint64_t tile = (uint64_t)BLK * V;
     float4* p4 = reinterpret_cast<float4*>(a.p);

@@ -41,6 +41,8 @@ cudaError_t run_arrive(const alsgd_sweep_buffers& b, uint32_t phase, cudaStream_
     a.seed_base[0] = b.snapshot;
     a.shared_base = BASE == kBaseShared;
     a.beta = 0.9f; a.eps = 0.7f; a.inv_n = 1.0f / (float)(K > 4 ? 8 : 4); a.cb = 0.9f; a.cn = 0.0f;
+    const bool pdl = (phase & ALSGD_SWEEP_LAUNCH_DEPENDENT) != 0;
+    phase &= ~ALSGD_SWEEP_LAUNCH_DEPENDENT;
     if (phase == ALSGD_SWEEP_PHASE_CYCLE) {
         a.flags = kDeltaZeroIn | kDeltaSkipStore | kReadM | kWriteM;
         a.boundary_mask = 1u << (K - 1);
@@ -51,7 +53,8 @@ cudaError_t run_arrive(const alsgd_sweep_buffers& b, uint32_t phase, cudaStream_
     cudaError_t e = grid_for(a.n, (uint64_t)V * BLK, &grid);
     if (e != cudaSuccess) return e;
     if (PERSIST) grid = resident_grid(kern, BLK, grid);
-    kern<<<grid, BLK, 0, s>>>(a);
+    e = launch_kernel(kern, grid, BLK, s, a, pdl);
+    if (e != cudaSuccess) return e;
     if (DIAG) {
         double* chunk_sum = a.diag_partial + (uint64_t)K * grid;
         diag_reduce1_kernel<<<dim3(kDiagChunks, K), kDiagBlock, 0, s>>>(a.diag_partial, grid, chunk_sum);
@@ -61,7 +64,7 @@ cudaError_t run_arrive(const alsgd_sweep_buffers& b, uint32_t phase, cudaStream_
 }
 
 template <int V, int BLK, int MINB, bool PERSIST>
-cudaError_t run_adamw(const alsgd_sweep_buffers& b, uint32_t, cudaStream_t s) {
+cudaError_t run_adamw(const alsgd_sweep_buffers& b, uint32_t phase, cudaStream_t s) {
     AdamArgs a{};
     a.p = b.adam_p; a.p_src = b.adam_p; a.m = b.adam_m; a.v = b.adam_v; a.g = b.adam_g; a.rep = b.adam_rep;
     a.seg_end = b.seg_end; a.seg_decay = b.seg_decay; a.n_seg = b.n_seg;
@@ -73,8 +76,7 @@ cudaError_t run_adamw(const alsgd_sweep_buffers& b, uint32_t, cudaStream_t s) {
     cudaError_t e = grid_for(a.n, (uint64_t)V * BLK, &grid);
     if (e != cudaSuccess) return e;
     if (PERSIST) grid = resident_grid(kern, BLK, grid);
-    kern<<<grid, BLK, 0, s>>>(a);
-    return cudaGetLastError();
+    return launch_kernel(kern, grid, BLK, s, a, (phase & ALSGD_SWEEP_LAUNCH_DEPENDENT) != 0);
 }
 
 // ---------------------------------------------------------------------------------------------------------

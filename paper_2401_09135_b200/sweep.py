@@ -92,7 +92,7 @@ def decay_segments(tensors, offsets, P):
     return ends, flags
 
 
-def run(n, select=None, reps=10, warmup=3, phase_for=None, log=None, segments=None):
+def run(n, select=None, reps=10, warmup=3, phase_for=None, log=None, segments=None, adam_phase=0):
     """Time every variant (or those select(v) accepts) on vectors of n elements.  Returns a list of dicts with
     the variant's fields, the phase, ms per launch and GB/s on the algorithmic bytes."""
     import torch
@@ -131,9 +131,9 @@ def run(n, select=None, reps=10, warmup=3, phase_for=None, log=None, segments=No
             continue
         if v["kind"] == KIND_ARRIVE:
             phase = phase_for(v) if phase_for else (PHASE_CYCLE if v["K"] == 8 else PHASE_MIDDLE)
-            bpp = arrive_bytes_per_param(v["K"], v["base_mode"], phase)
+            bpp = arrive_bytes_per_param(v["K"], v["base_mode"], phase & 0xFF)
         else:
-            phase, bpp = 0, ADAMW_BYTES_PER_PARAM
+            phase, bpp = adam_phase, ADAMW_BYTES_PER_PARAM
         for _ in range(warmup):
             rc = L.alsgd_sweep_launch(v["index"], C.byref(b), phase, stream)
             if rc != 0:
