@@ -89,14 +89,16 @@ def init_theta(P, offsets, seed):
 
 
 def run(speeds, N, outer_lr=0.7, beta=0.9, H=20, dylu=True, tau_grace=0.0, total_local_steps=4000, batch=64,
-        lr_max=3e-3, lr_min=1e-5, warmup=50, seed=7, buffered=False, device=0, log_every=0, sample_shards=True):
+        lr_max=3e-3, lr_min=1e-5, warmup=50, seed=7, buffered=False, sgdm=False, device=0, log_every=0,
+        sample_shards=True):
     """Asynchronous Local-SGD on the toy task through the library.  Returns (validation loss, accuracy,
     number of server updates, final theta as a CPU tensor)."""
     torch.cuda.set_device(device)
     dev = torch.device("cuda", device)
     W = len(speeds)
     tensors = mlp_tensors()
-    ctx = B.Context(tensors, W, N, beta, outer_lr, adam=(0.9, 0.95, 1e-8, 0.1), align_elems=4, device=device, buffered=buffered)
+    ctx = B.Context(tensors, W, N, beta, outer_lr, adam=(0.9, 0.95, 1e-8, 0.1), align_elems=4, device=device, buffered=buffered,
+                    sgdm=sgdm)
     P, offsets = ctx.P, ctx.offsets
     shards, val = make_data(W, 4000, seed, dev)
     ctx.alsgd_set_global(init_theta(P, offsets, seed).numpy())
@@ -162,14 +164,16 @@ def main():
     rows = [
         ("synchronous (equal speeds, one window, N = 4)", dict(speeds=[1.0] * 4, N=4, dylu=False)),
         ("async Nesterov (N = 1), heterogeneous", dict(speeds=hetero, N=1, dylu=False)),
+        ("async SGD Momentum at every arrival (N = 1), heterogeneous", dict(speeds=hetero, N=1, dylu=False, sgdm=True)),
+        ("async plain outer SGD (SGD Momentum with beta = 0), heterogeneous", dict(speeds=hetero, N=1, dylu=False, sgdm=True, beta=0.0)),
         ("async buffered (N = 4), heterogeneous", dict(speeds=hetero, N=4, dylu=False, buffered=True)),
         ("async Delayed Nesterov (N = 4), heterogeneous", dict(speeds=hetero, N=4, dylu=False)),
         ("async Delayed Nesterov + DyLU, grace 0.5", dict(speeds=hetero, N=4, dylu=True, tau_grace=0.5)),
     ]
-    print(f"{'setting':58s} {'val loss':>9s} {'accuracy':>9s} {'server updates':>15s}")
+    print(f"{'setting':70s} {'val loss':>9s} {'accuracy':>9s} {'server updates':>15s}")
     for name, kw in rows:
         vloss, acc, updates, _ = run(total_local_steps=args.steps, **kw)
-        print(f"{name:58s} {vloss:9.4f} {acc:9.4f} {updates:15d}")
+        print(f"{name:70s} {vloss:9.4f} {acc:9.4f} {updates:15d}")
 
 
 if __name__ == "__main__":
