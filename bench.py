@@ -399,10 +399,10 @@ def main_ours(args, rank, world, local_rank):
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
-            n_cpu = P // 8
+            n_cpu = P // 4
             cpu_order = [order[0]]
             v, dt, p = run_oracle(n_cpu, cpu_order, steps, 0, 1)
-            sample = f"first {n_cpu} elements (an eighth) of the layout, one step: {steps[cpu_order[0]]} inner AdamW steps + 1 arrival with re-seed"
+            sample = f"first {n_cpu} elements (a quarter) of the layout, one step: {steps[cpu_order[0]]} inner AdamW steps + 1 arrival with re-seed"
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt, "sample": sample}
             cores = os.cpu_count() or 1
             vn, dtn = run_oracle_all_cores(n_cpu, cpu_order[0], steps[cpu_order[0]], cores)
