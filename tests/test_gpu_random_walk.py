@@ -16,11 +16,24 @@ pytestmark = pytest.mark.gpu
                                                           (3, False, True, 0.0, 2), (4, False, False, 0.125, 4),
                                                           (5, False, False, 0.0, 1), (6, True, True, 0.0, 5)])
 def test_random_walk(seed, pg_current, buffered, c, N):
+    walk(seed, pg_current, buffered, c, N)
+
+
+@pytest.mark.parametrize("seed,pg_current,N,kw", [(7, False, 3, dict(sgdm=True)), (8, True, 1, dict(sgdm=True)),
+                                                  (9, False, 4, dict(stable_ptrs=True)), (10, True, 2, dict(stable_ptrs=True, buffered=True)),
+                                                  (11, False, 8, dict(W=11)), (12, True, 3, dict(W=9, stable_ptrs=True))])
+def test_random_walk_outer_modes_stable_pointers_and_large_batches(seed, pg_current, N, kw):
+    """The same walk with the SGD Momentum outer step, with permanent pointers, and with enough workers for
+    batches of eight and batches split over launches."""
+    walk(seed, pg_current, kw.pop("buffered", False), 0.0, N, **kw)
+
+
+def walk(seed, pg_current, buffered, c, N, sgdm=False, stable_ptrs=False, W=6, steps=160):
     r = np.random.default_rng(seed)
     tensors = synth.ragged_tensors()
-    W = 6
     align = int(r.choice([1, 4, 8]))
-    pair = Pair(tensors, W, N, 0.9, 0.7, c=c, pg_current=pg_current, align=align, buffered=buffered)
+    pair = Pair(tensors, W, N, 0.9, 0.7, c=c, pg_current=pg_current, align=align, buffered=buffered, sgdm=sgdm,
+                stable_ptrs=stable_ptrs)
     P = pair.P
     pair.set_global(synth.theta0(tensors, pair.offsets, P, synth.SEED + seed))
     dispatched = set()
@@ -32,7 +45,7 @@ def test_random_walk(seed, pg_current, buffered, c, N):
         return synth.zero_padding(synth.normal_vec(P, std, synth.SEED + seed, stream, sub=int(r.integers(0, 1 << 30))),
                                   tensors, pair.offsets)
 
-    for step in range(160):
+    for step in range(steps):
         op = r.choice(["pull", "adam", "adam16", "arrive", "arrive", "set", "get", "ckpt"],
                       p=[0.12, 0.25, 0.08, 0.15, 0.15, 0.08, 0.09, 0.08])
         if op == "pull" or not dispatched:
@@ -79,7 +92,7 @@ def test_random_walk(seed, pg_current, buffered, c, N):
         elif op == "ckpt":
             image = pair.ctx.alsgd_export_state()
             fresh = B.Context(tensors, W, N, 0.9, 0.7, c=c, pg_base=B.PG_CURRENT if pg_current else B.PG_DISPATCH,
-                              align_elems=align, buffered=buffered)
+                              align_elems=align, buffered=buffered, sgdm=sgdm, stable_ptrs=stable_ptrs)
             fresh.alsgd_import_state(image)
             pair.ctx.close()
             pair.ctx = fresh
