@@ -56,7 +56,8 @@ typedef struct alsgd_sweep_buffers {
     uint32_t reserved;
     double* diag_scratch;     /* 8 * (n / 256 + 66) doubles (diag variants only) */
     double* diag_out;         /* 8 doubles */
-    unsigned int* diag_flags; /* 8 words */
+    unsigned int* diag_flags; /* 8 words, zero before the first launch */
+    unsigned int* diag_state; /* 16 words, zero before the first launch: 8 counters of the reduction, then the 8 flags it hands out */
 } alsgd_sweep_buffers;
 
 /* Position in the Delayed Nesterov cycle an arrival pass is timed at. */

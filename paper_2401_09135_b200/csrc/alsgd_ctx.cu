@@ -104,7 +104,7 @@ struct alsgd_ctx {
     uint32_t n_seg = 0;
     double* gnorm2 = nullptr;
     double* diag_partial = nullptr;
-    unsigned int* nonfinite = nullptr;
+    unsigned int* nonfinite = nullptr;      // [0, 8): flags the pass ORs into; [8, 16): flags handed out; [16, 24): tickets
     unsigned int* guard_word = nullptr;   // debug build: violations recorded by the kernels' bounds checks
     float* theta = nullptr;
     float* mom = nullptr;
@@ -142,7 +142,7 @@ uint64_t carve(alsgd_ctx* c, void* arena, uint64_t P, const alsgd_config& cfg, u
     uint32_t* seg_decay = k.take<uint32_t>(n_seg);
     double* gn = k.take<double>(kMaxArrivals);
     double* gpart = k.take<double>(diag_partial_count(P));
-    unsigned int* nf = k.take<unsigned int>(kMaxArrivals);
+    unsigned int* nf = k.take<unsigned int>(3 * kMaxArrivals);
     unsigned int* gw = k.take<unsigned int>(1);
     float* theta = k.take<float>(P);
     float* mom = k.take<float>(P);
@@ -350,7 +350,7 @@ int alsgd_init(alsgd_ctx** out, const alsgd_tensor_desc* tensors, uint32_t n, ui
         // The segment tables live in pageable host vectors that die with this scope.
         if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->gnorm2, 0, sizeof(double) * kMaxArrivals, c->stream);
-        if (e == cudaSuccess) e = cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * kMaxArrivals, c->stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * 3 * kMaxArrivals, c->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->guard_word, 0, sizeof(unsigned int), c->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->theta, 0, sizeof(float) * P, c->stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->mom, 0, sizeof(float) * P, c->stream);
@@ -593,6 +593,7 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
         ArriveArgs a{};
         a.theta = c->theta; a.delta = c->delta; a.mom = c->mom;
         a.gnorm2 = c->gnorm2; a.diag_partial = c->diag_partial; a.nonfinite = c->nonfinite;
+        a.nonfinite_out = c->nonfinite + kMaxArrivals; a.diag_ticket = c->nonfinite + 2 * kMaxArrivals;
         a.n = c->P;
         a.n_arr = kk;
         a.beta = c->cfg.beta; a.eps = c->cfg.outer_lr; a.inv_n = c->inv_n; a.cb = c->cb; a.cn = c->cn;
@@ -632,16 +633,13 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
             seeded = ns;
             snapshot_written = true;
         }
-        if (diag) {
-            ALSGD_STEP(cudaMemsetAsync(c->nonfinite, 0, sizeof(unsigned int) * kMaxArrivals, c->stream));
-        }
         ALSGD_STEP(launch_arrive(a, current, diag, extended, c->stream));
         enqueued = true;
         if (diag && info) {
             double nb[kMaxArrivals];
             unsigned int fb[kMaxArrivals];
             ALSGD_STEP(cudaMemcpyAsync(nb, c->gnorm2, sizeof(double) * kk, cudaMemcpyDeviceToHost, c->stream));
-            ALSGD_STEP(cudaMemcpyAsync(fb, c->nonfinite, sizeof(unsigned int) * kk, cudaMemcpyDeviceToHost, c->stream));
+            ALSGD_STEP(cudaMemcpyAsync(fb, c->nonfinite + kMaxArrivals, sizeof(unsigned int) * kk, cudaMemcpyDeviceToHost, c->stream));
             ALSGD_STEP(cudaStreamSynchronize(c->stream));
             for (uint32_t j = 0; j < kk; ++j) { norms[active[j0 + j]] = nb[j]; bads[active[j0 + j]] = fb[j]; }
         }

@@ -45,8 +45,18 @@ cudaError_t launch_arrive_k(const ArriveArgs& a, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     if (DIAG && K > 0) {
         double* chunk_sum = a.diag_partial + (uint64_t)K * grid;        // behind the K x grid partials
-        diag_reduce1_kernel<<<dim3(kDiagChunks, K), kDiagBlock, 0, s>>>(a.diag_partial, grid, chunk_sum);
-        diag_reduce2_kernel<<<1, 32, 0, s>>>(chunk_sum, K, a.gnorm2);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kDiagChunks, K);
+        cfg.blockDim = dim3(kDiagBlock);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, diag_reduce_kernel, (const double*)a.diag_partial, (uint32_t)grid, chunk_sum, a.gnorm2,
+                               a.nonfinite, a.nonfinite_out, a.diag_ticket);
+        if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();
 }

@@ -42,7 +42,9 @@ struct ArriveArgs {
     uint16_t* seed_rep[kMaxSeeds];    // may be null
     double* gnorm2;                   // out: kMaxArrivals squared norms (written by the reduction that follows the pass)
     double* diag_partial;             // scratch: one double per block per arrival, diag_partial_count(n) entries
-    unsigned int* nonfinite;          // scratch: kMaxArrivals flags, zeroed by the caller
+    unsigned int* nonfinite;          // scratch: kMaxArrivals flags the pass ORs into; zero on entry, put back to zero by the reduction
+    unsigned int* nonfinite_out;      // out: kMaxArrivals flags (written by the reduction that follows the pass)
+    unsigned int* diag_ticket;        // scratch: kMaxArrivals counters of the reduction; zero between launches
     uint64_t n;                       // elements
     uint32_t n_arr;
     uint32_t n_seed;

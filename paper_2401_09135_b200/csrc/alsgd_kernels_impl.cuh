@@ -430,14 +430,21 @@ __global__ void __launch_bounds__(BLK, MINB) arrive_kernel(const __grid_constant
     }
 }
 
-// Two-stage, fixed-order sum of the per-block partials partial[arrival][block].
-// Stage 1: block (r, j) adds the r-th of kDiagChunks contiguous chunks of arrival j's partials.
+// Fixed-order sum of the per-block partials partial[arrival][block], in one launch that follows the pass.
+// Block (r, j) adds the r-th of kDiagChunks contiguous chunks of arrival j's partials; the block of an arrival
+// that finishes last (a ticket counter per arrival) adds the kDiagChunks chunk sums in index order, hands out the
+// arrival's norm and non-finite flag, and puts flag and counter back to zero for the next pass.  The order of
+// every addition is fixed, so the same inputs give the same bits whichever block happens to be last.
 constexpr int kDiagChunks = 64;
 constexpr int kDiagBlock = 256;
 
-__global__ void __launch_bounds__(kDiagBlock) diag_reduce1_kernel(const double* __restrict__ partial, uint32_t n_blocks,
-                                                                  double* __restrict__ chunk_sum) {
+__global__ void __launch_bounds__(kDiagBlock) diag_reduce_kernel(const double* __restrict__ partial, uint32_t n_blocks,
+                                                                 double* chunk_sum, double* __restrict__ gnorm2_out,
+                                                                 unsigned int* flag_acc, unsigned int* flag_out,
+                                                                 unsigned int* ticket) {
+    grid_dependency_sync();
     __shared__ double lane_sum[kDiagBlock];
+    __shared__ bool last;
     const uint32_t r = blockIdx.x, j = blockIdx.y;
     const uint32_t per = (n_blocks + kDiagChunks - 1) / kDiagChunks;
     const uint32_t lo = min(r * per, n_blocks), hi = min(lo + per, n_blocks);
@@ -450,16 +457,18 @@ __global__ void __launch_bounds__(kDiagBlock) diag_reduce1_kernel(const double* 
         double t = 0.0;
         for (int i = 0; i < kDiagBlock; ++i) t += lane_sum[i];
         chunk_sum[j * kDiagChunks + r] = t;
+        __threadfence();                                        // the chunk sum is visible before the ticket is taken
+        last = atomicAdd(ticket + j, 1u) == (unsigned)kDiagChunks - 1u;
     }
-}
-
-// Stage 2: thread j adds arrival j's chunk sums in order.
-__global__ void diag_reduce2_kernel(const double* __restrict__ chunk_sum, uint32_t K, double* __restrict__ out) {
-    const uint32_t j = threadIdx.x;
-    if (j < K) {
+    __syncthreads();
+    if (last && threadIdx.x == 0) {
+        __threadfence();
+        const volatile double* cs = chunk_sum + j * kDiagChunks;   // written by other blocks: read past L1
         double t = 0.0;
-        for (int r = 0; r < kDiagChunks; ++r) t += chunk_sum[j * kDiagChunks + r];
-        out[j] = t;
+        for (int q = 0; q < kDiagChunks; ++q) t += cs[q];
+        gnorm2_out[j] = t;
+        flag_out[j] = atomicExch(flag_acc + j, 0u) ? 1u : 0u;
+        ticket[j] = 0u;
     }
 }
 

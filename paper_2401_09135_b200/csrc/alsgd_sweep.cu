@@ -57,8 +57,8 @@ cudaError_t run_arrive(const alsgd_sweep_buffers& b, uint32_t phase, cudaStream_
     if (e != cudaSuccess) return e;
     if (DIAG) {
         double* chunk_sum = a.diag_partial + (uint64_t)K * grid;
-        diag_reduce1_kernel<<<dim3(kDiagChunks, K), kDiagBlock, 0, s>>>(a.diag_partial, grid, chunk_sum);
-        diag_reduce2_kernel<<<1, 32, 0, s>>>(chunk_sum, K, a.gnorm2);
+        diag_reduce_kernel<<<dim3(kDiagChunks, K), kDiagBlock, 0, s>>>(a.diag_partial, grid, chunk_sum, a.gnorm2, a.nonfinite,
+                                                                       b.diag_state + 8, b.diag_state);
     }
     return cudaGetLastError();
 }

@@ -28,7 +28,7 @@ class Buffers(C.Structure):
                 ("adam_p", C.c_void_p), ("adam_m", C.c_void_p), ("adam_v", C.c_void_p), ("adam_g", C.c_void_p),
                 ("adam_rep", C.c_void_p), ("seg_end", C.c_void_p), ("seg_decay", C.c_void_p),
                 ("n_seg", C.c_uint32), ("reserved", C.c_uint32),
-                ("diag_scratch", C.c_void_p), ("diag_out", C.c_void_p), ("diag_flags", C.c_void_p)]
+                ("diag_scratch", C.c_void_p), ("diag_out", C.c_void_p), ("diag_flags", C.c_void_p), ("diag_state", C.c_void_p)]
 
 
 _lib = None
@@ -124,6 +124,7 @@ def run(n, select=None, reps=10, warmup=3, phase_for=None, log=None, segments=No
     b.diag_out = hold(torch.zeros(8, device=dev, dtype=torch.float64))
     keep_flags = torch.zeros(8, device=dev, dtype=torch.int32)
     b.diag_flags = hold(keep_flags)
+    b.diag_state = hold(torch.zeros(16, device=dev, dtype=torch.int32))
     stream = torch.cuda.current_stream().cuda_stream
     rows = []
     for v in variants():

@@ -35,10 +35,11 @@ def _buffers(n, seed):
     t["diag_scratch"] = torch.zeros(8 * (n // 256 + 66), device=dev, dtype=torch.float64)
     t["diag_out"] = torch.zeros(8, device=dev, dtype=torch.float64)
     t["diag_flags"] = torch.zeros(8, device=dev, dtype=torch.int32)
+    t["diag_state"] = torch.zeros(16, device=dev, dtype=torch.int32)
     b = sweep.Buffers()
     b.n = n
     for name in ("theta", "delta", "mom", "snapshot", "adam_p", "adam_m", "adam_v", "adam_g", "adam_rep", "seg_end",
-                 "seg_decay", "diag_scratch", "diag_out", "diag_flags"):
+                 "seg_decay", "diag_scratch", "diag_out", "diag_flags", "diag_state"):
         setattr(b, name, t[name].data_ptr())
     for j in range(8):
         b.p[j], b.base[j], b.rep[j] = t[f"p{j}"].data_ptr(), t[f"base{j}"].data_ptr(), t[f"rep{j}"].data_ptr()
@@ -94,5 +95,5 @@ def test_every_arrival_shape_gives_the_same_bits(phase):
             if ref[key][1] is None:
                 ref[key] = (ref[key][0], norms)
             assert torch.allclose(norms, ref[key][1], rtol=1e-6, atol=0.0), v
-            assert not t["diag_flags"][:K].any()
+            assert not t["diag_flags"][:K].any() and not t["diag_state"].any()
     assert len(ref) >= 7
