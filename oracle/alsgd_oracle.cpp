@@ -14,6 +14,8 @@
 //   orc_adamw       hand case, sign-step property, pure-decay geometric sequence, undecayed tensors.
 //                   The paper prints no AdamW formula; the variant is the textbook decoupled one.
 //   orc_bf16_rne    exhaustive check against nearest-neighbour search over a strided 2^32 sweep.
+//   orc_pg_norm2    hand values against the dispatch snapshot and against the running theta (decoy snapshot), the
+//                   second arrival of a batch against theta after the first, NaN / Inf flagged.
 //   orc_dylu        Eq. 6 values for speeds 1:1.5:2:3, H = 50.
 //   orc_lr_at       Eq. 3 end points and clamps.
 //   orc_schedule    Algorithm 2 + Algorithm 5 on hand timelines (Fig. 3 description).
