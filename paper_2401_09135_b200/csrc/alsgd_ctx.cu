@@ -130,6 +130,9 @@ struct alsgd_ctx {
     // Set when a call failed after some of its launches were already enqueued: the device state is then
     // ahead of the host bookkeeping, and every later state-changing call is refused.
     bool poisoned = false;
+    // Consecutive whole-vector launches walk the vector in opposite directions, so that what the previous launch
+    // touched last (and the L2 still holds) is what the next one touches first.
+    uint32_t direction = 0;
     uintptr_t arena_lo = 0, arena_hi = 0;
 };
 
@@ -421,6 +424,7 @@ int alsgd_pull(alsgd_ctx* c, uint32_t worker) {
     a.n_arr = 0;
     a.n_seed = 1;
     fill_guard(c, a.guard);
+    a.reverse = (c->direction ^= 1u);
     const int slot = pick_slot(c, &worker, 1);
     fill_seed(c, a, 0, worker, slot >= 0 ? c->slot_ptr[slot] : nullptr);
     DeviceGuard g(c->cfg.device);
@@ -466,6 +470,7 @@ int adamw_impl(alsgd_ctx* c, uint32_t worker, const void* grads, bool bf16, int 
         return launch_adamw(a, grads_is_device != 0, c->stream);
     };
     if (grads_is_device) {
+        a.reverse = (c->direction ^= 1u);
         ALSGD_CUDA(c, launch_range(0, c->P, grads));
     } else {
         // Chunked: copy chunk i on the copy stream, run the step on it on the context's stream as soon as
@@ -602,6 +607,7 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
         a.beta2 = sgdm ? c->cfg.beta : c->cfg.beta * c->cfg.beta;
         a.one_plus_beta = sgdm ? 1.0f : 1.0f + c->cfg.beta;
         fill_guard(c, a.guard);
+        a.reverse = (c->direction ^= 1u);
         bool any_boundary = false, last_boundary = false;
         a.shared_base = current ? 0u : 1u;
         for (uint32_t j = 0; j < kk; ++j) {
@@ -655,6 +661,7 @@ int arrive_impl(alsgd_ctx* c, const uint32_t* ids, uint32_t k, uint32_t flags, c
             ArriveArgs a{};
             a.theta = c->theta; a.n = c->P; a.n_seed = ns;
             fill_guard(c, a.guard);
+            a.reverse = (c->direction ^= 1u);
             for (uint32_t s = 0; s < ns; ++s) {
                 fill_seed(c, a, s, ids[at + s], snapshot_written ? nullptr : snapshot);
                 snapshot_written = true;

@@ -57,6 +57,7 @@ struct ArriveArgs {
     float beta2, one_plus_beta;       // momentum and gradient weights of the buffered step: beta*beta and 1+beta
                                       // (Eq. 4), or beta and 1 (SGD Momentum); each one fp32 operation
     uint32_t shared_base;             // 1: every arrival was dispatched with the snapshot base[0]
+    uint32_t reverse;                 // 1: blocks take the tiles from the last to the first
     DebugGuard guard;
 };
 
@@ -74,6 +75,7 @@ struct AdamArgs {
     uint64_t n;                // elements in this launch
     uint64_t seg_base;         // flat index of this launch's first element (segment ends are flat indices)
     float b1, b2, omb1, omb2, bc1, bc2, eps, lr, wd;
+    uint32_t reverse;          // 1: blocks take the tiles from the last to the first
     DebugGuard guard;
 };
 
