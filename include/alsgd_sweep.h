@@ -68,6 +68,10 @@ typedef struct alsgd_sweep_buffers {
  * kernel of the stream drains and wait, before their first memory access, for its completion).  Register variants only. */
 #define ALSGD_SWEEP_LAUNCH_DEPENDENT 0x100u
 
+/* OR-ed into `phase` (AdamW variants): walk the vector in the opposite direction of the previous launch, so that the
+ * state the previous launch touched last, which L2 still holds, is touched first. */
+#define ALSGD_SWEEP_LAUNCH_ALTERNATE 0x200u
+
 int alsgd_sweep_count(void);
 /* idx in [0, count).  Returns 0, or -1 for a bad index or null pointer. */
 int alsgd_sweep_describe(int idx, alsgd_sweep_variant* out);

@@ -72,7 +72,7 @@ cudaError_t run_adamw(const alsgd_sweep_buffers& b, uint32_t phase, cudaStream_t
     a.b1 = 0.9f; a.b2 = 0.95f; a.omb1 = 1.0f - a.b1; a.omb2 = 1.0f - a.b2;
     a.bc1 = 0.65f; a.bc2 = 0.4f; a.eps = 1e-8f; a.lr = 1e-3f; a.wd = 0.1f;
     static unsigned flip = 0;
-    if (phase & 0x200u) a.reverse = (flip++) & 1u;               // experiment: alternate the tile order launch by launch
+    if (phase & ALSGD_SWEEP_LAUNCH_ALTERNATE) a.reverse = (flip++) & 1u;
     auto kern = adamw_kernel<V, BLK, MINB, false, PERSIST>;
     unsigned grid = 1;
     cudaError_t e = grid_for(a.n, (uint64_t)V * BLK, &grid);
