@@ -44,8 +44,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter from the committed ncu captures
 # (profiles/), valid only for the kernel source they were taken from.
 NCU_TRAFFIC = {
-    "src_sha256": "689f949c0d89e6df91158617ec21ba17fad0944cdaad8bae05035e1c3c2167a9",
-    "adamw_bytes_per_param": 28.91,     # ncu capture at P = 50.3M elements (profiles/adamw_kernel_flat48M.md), scaled by P
+    "src_sha256": "a38ecdfa04e6e4fcc6f8673ea58393910425528c24765c0bd2fe7ff66de9691a",
+    "adamw_bytes_per_param": 28.90,     # ncu capture at P = 50.3M elements (profiles/adamw_kernel_flat48M.md), scaled by P
     "arrive_bytes_per_param": 28.90,    # same capture, K = 1, average over one Delayed-Nesterov cycle
 }
 
