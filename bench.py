@@ -562,7 +562,11 @@ def main_shape_sweep(args):
         assert P == n
         segments = sweep.decay_segments(tensors, offsets, P)
     kinds = {"all": None, "adamw": sweep.KIND_ADAMW, "arrive": sweep.KIND_ARRIVE}[args.sweep_kind]
-    rows = sweep.run(n, reps=args.sweep_reps, warmup=3, segments=segments,
+    # --sweep-product-launch: launch the way the library does (programmatic dependent launch; AdamW walking the vector
+    # in the opposite direction of the previous launch) instead of plain identical launches
+    dep, alt = (0x100, 0x200) if args.sweep_product_launch else (0, 0)
+    rows = sweep.run(n, reps=args.sweep_reps, warmup=3, segments=segments, adam_phase=dep | alt,
+                     phase_for=(lambda v: (sweep.PHASE_CYCLE if v["K"] == 8 else sweep.PHASE_MIDDLE) | dep) if dep else None,
                      select=(lambda v: v["kind"] == kinds) if kinds is not None else None,
                      log=(lambda r: print(json.dumps(r), file=sys.stderr, flush=True)) if args.verbose else None)
     best = {}
@@ -572,7 +576,7 @@ def main_shape_sweep(args):
         key = ("adamw" if r["kind"] == sweep.KIND_ADAMW else f"arrive K={r['K']} base={sweep.BASE_NAMES[r['base_mode']]}") + (" diag" if r["diag"] else "")
         if key not in best or r["gbs"] > best[key]["gbs"]:
             best[key] = r
-    print(json.dumps({"elements": n, "reps": args.sweep_reps, "peak_gbs": peak, "peak_source": f"of {which}",
+    print(json.dumps({"elements": n, "reps": args.sweep_reps, "product_launch": bool(args.sweep_product_launch), "peak_gbs": peak, "peak_source": f"of {which}",
                       "unit": "GB/s on algorithmic bytes", "best": best, "rows": rows}), flush=True)
 
 
@@ -694,6 +698,8 @@ def main():
     ap.add_argument("--sweep-elems", type=int, default=109_549_056)
     ap.add_argument("--sweep-reps", type=int, default=10)
     ap.add_argument("--sweep-kind", choices=["all", "adamw", "arrive"], default="all")
+    ap.add_argument("--sweep-product-launch", action="store_true",
+                    help="shape sweep with dependent launches and alternating direction, as the library launches")
     ap.add_argument("--verbose", action="store_true")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
