@@ -362,7 +362,9 @@ def main_ours(args, rank, world, local_rank):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": WORKLOAD, "P": P, "H": H, "speeds": SPEEDS, "dylu_steps": steps,
                        "step": "one scheduled arrival: DyLU inner AdamW steps of the arriving worker + DN arrival with fused re-seed",
-                       "l2": "every launch streams 3.3-3.7 GB (inputs larger than the 126 MB L2); no flush needed",
+                       "l2": "every launch streams 3.3-3.7 GB (inputs larger than the 126 MB L2); no flush. By design consecutive launches walk the "
+                             "vectors in opposite directions, so a step re-touches first what the previous step of the same worker left in L2 "
+                             "(worth 1.3 % at this size)",
                        "multi_gpu": "each rank holds its own 110M-element range of an N-times larger vector; no exchange"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
