@@ -240,3 +240,43 @@ def test_schedule_stops_at_t_max_local_updates():
     w, t, b = oracle.schedule(dur, [10, 20], tau_grace=0.0, t_max=45, max_arrivals=100)
     # t_local after each arrival: 10 (w0@1), then a tie at 2 (w0, w1) -> 20, 40; w0@3 -> 50 >= 45 stops
     assert w == [0, 0, 1, 0]
+
+
+def test_schedule_invariants_on_random_timelines():
+    """What Algorithm 2 with Algorithm 5 guarantees on any input, checked on the oracle's output alone: a window
+    is opened by the earliest pending completion; everything completing within tau_grace of it joins, in
+    (time, id) order, and nothing that completes within the window is left out; the workers of a window restart
+    together at tau_sync + tau_grace, so a worker's next completion is that restart plus its next duration."""
+    r = np.random.default_rng(11)
+    for case in range(60):
+        W = int(r.integers(2, 8))
+        R = 12
+        dur = r.uniform(0.5, 3.0, size=(W, R))
+        if case % 3 == 0:
+            dur = np.round(dur * 2) / 2                     # many exact ties
+        grace = float(r.choice([0.0, 0.25, 1.0, 4.0]))
+        w, t, b = oracle.schedule(dur, [1] * W, grace, 10 ** 9, 5 * W)
+        done = [dur[u, 0] for u in range(W)]                # current completion time of every worker's job
+        rounds = [0] * W
+        pending = set(range(W))
+        i = 0
+        while i < len(w):
+            j = i
+            while j < len(w) and b[j] == b[i]:
+                j += 1
+            batch = list(zip(w[i:j], t[i:j]))
+            full = j < len(w)                               # the last window may be cut by max_arrivals
+            first_w, tau_sync = batch[0]
+            assert tau_sync == min(done[u] for u in pending)                     # earliest pending opens it
+            assert all(done[u] == tu for u, tu in batch)                         # reported time = completion time
+            assert batch == sorted(batch, key=lambda x: (x[1], x[0]))            # (time, id) order
+            assert all(tu - tau_sync <= grace for _, tu in batch)                # inside the window
+            if full:
+                left = pending - {u for u, _ in batch}
+                assert all(not (done[u] - tau_sync <= grace) for u in left)      # nobody inside was left out
+            restart = tau_sync + grace
+            for u, _ in batch:
+                rounds[u] += 1
+                if rounds[u] < R:
+                    done[u] = restart + dur[u, rounds[u]]
+            i = j

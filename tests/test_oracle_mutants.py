@@ -31,7 +31,7 @@ BF16_PINS = [misc.test_bf16_named_values, misc.test_bf16_every_high_half_at_the_
 HOST_PINS = [misc.test_shard_sampling_eq2, misc.test_dylu_values, misc.test_lr_schedule_endpoints_and_clamps, misc.test_poly_weight,
              misc.test_schedule_grace_window_timeline, misc.test_schedule_equal_speeds_behave_synchronously,
              misc.test_schedule_zero_grace_distinct_times_gives_singletons_in_time_order,
-             misc.test_schedule_stops_at_t_max_local_updates]
+             misc.test_schedule_stops_at_t_max_local_updates, misc.test_schedule_invariants_on_random_timelines]
 VAR_PINS = [var.test_buffered_hand_trace, var.test_buffered_with_N1_is_plain_nesterov_and_matches_dn_at_cycle_ends,
             var.test_delay_compensation_hand_case_and_zero_drift, var.test_weighted_arrival_hand_case_and_homogeneity,
             var.test_poly_weights_and_threshold_bookkeeping, var.test_delay_compensation_comes_before_the_staleness_weight,
@@ -71,6 +71,10 @@ MUTANTS = [
     ("grace test strict", "completed_time[w] - tau_sync <= tau_grace", "completed_time[w] - tau_sync < tau_grace", None, HOST_PINS),
     ("restart without the grace period", "const double restart = tau_sync + tau_grace;", "const double restart = tau_sync;", None, HOST_PINS),
     ("t_local not counted", "t_local += local_updates[w];", "t_local += 0;", None, HOST_PINS),
+    ("workers of a window restart at their own completion, not together",
+     "completed_time[u] = restart + durations[(uint64_t)u * n_rounds + round[u]];",
+     "completed_time[u] = completed_time[u] + tau_grace + durations[(uint64_t)u * n_rounds + round[u]];", None, HOST_PINS),
+    ("window opened by the latest pending completion", "completed_time[u] < completed_time[w]) w = u;", "completed_time[u] > completed_time[w]) w = u;", None, HOST_PINS),
     ("shard gap sign", "const double gap = size_share - learned_share;", "const double gap = learned_share - size_share;", None, HOST_PINS),
     ("shard gap not clipped at zero", "probs[i] = gap > 0.0 ? gap : 0.0;", "probs[i] = gap > 0.0 ? gap : -gap;", None, HOST_PINS),
     ("shard probabilities not normalised", "probs[i] = norm > 0.0 ? probs[i] / norm : sizes[i] / total_size;", "probs[i] = norm > 0.0 ? probs[i] : sizes[i] / total_size;", None, HOST_PINS),
