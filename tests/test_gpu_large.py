@@ -66,3 +66,38 @@ def test_vectors_beyond_32_bit_offsets(P, need_gib):
     ctx.close()
     del grads, ctx
     torch.cuda.empty_cache()
+
+
+def test_110m_norms_of_batches_of_eight_against_the_oracle_on_the_full_vectors():
+    """The diagnostics in the launch configuration the benchmark times (110M elements, eight arrivals in one pass:
+    213 963 blocks, one partial per block per arrival, one reduction launch): every arrival's squared norm against
+    the oracle's double-precision sum over the complete vectors, first with eight distinct dispatch snapshots, then
+    with one shared snapshot, and a non-finite entry in the very last element."""
+    import oracle
+    tensors = synth.layout_110m()
+    W = 8
+    ctx = B.Context(tensors, W, 8, 0.9, 0.7)
+    P = ctx.P
+    ctx.alsgd_set_global(synth.theta0(tensors, ctx.offsets, P, synth.SEED + 31))
+    for w in range(W):
+        ctx.alsgd_pull(w)
+    z = [torch.from_numpy(synth.normal_vec(P, 1e-3 * (i + 1), synth.SEED + 31, synth.STREAM_DELTA, sub=i)).cuda() for i in range(2)]
+    for rnd in range(2):
+        ids = [3, 0, 7, 1, 6, 2, 5, 4] if rnd == 0 else [6, 4, 0, 2, 7, 5, 3, 1]
+        want = []
+        for j, w in enumerate(ids):
+            v = ctx.alsgd_worker_state_ptrs(w)
+            v["p"].sub_(z[(w + rnd) % 2])
+            if rnd == 1 and j == 5:
+                v["p"][P - 1] = float("inf")
+            base, p = v["base"].cpu().numpy(), v["p"].cpu().numpy()
+            want.append(oracle.pg_norm2(base, base, p))
+        bases = {ctx.alsgd_worker_state_ptrs(w)["base"].data_ptr() for w in ids}
+        assert len(bases) == (8 if rnd == 0 else 1)
+        info = ctx.alsgd_arrive(ids, B.ARRIVE_RESEED | B.ARRIVE_NORM | B.ARRIVE_NANCHECK)
+        for j, (got, (norm, bad)) in enumerate(zip(info, want)):
+            assert got["nonfinite"] == bad == (1 if (rnd == 1 and j == 5) else 0)
+            if not bad:
+                assert abs(got["gnorm2"] - norm) <= 1e-6 * norm, (rnd, j, got["gnorm2"], norm)
+    ctx.alsgd_sync()
+    ctx.close()
