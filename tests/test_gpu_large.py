@@ -77,10 +77,12 @@ def test_110m_norms_of_batches_of_eight_against_the_oracle_on_the_full_vectors()
     tensors = synth.layout_110m()
     W = 8
     ctx = B.Context(tensors, W, 8, 0.9, 0.7)
+    plain = B.Context(tensors, W, 8, 0.9, 0.7)               # the same run without diagnostics: same bits expected
     P = ctx.P
-    ctx.alsgd_set_global(synth.theta0(tensors, ctx.offsets, P, synth.SEED + 31))
-    for w in range(W):
-        ctx.alsgd_pull(w)
+    for c in (ctx, plain):
+        c.alsgd_set_global(synth.theta0(tensors, ctx.offsets, P, synth.SEED + 31))
+        for w in range(W):
+            c.alsgd_pull(w)
     z = [torch.from_numpy(synth.normal_vec(P, 1e-3 * (i + 1), synth.SEED + 31, synth.STREAM_DELTA, sub=i)).cuda() for i in range(2)]
     for rnd in range(2):
         ids = [3, 0, 7, 1, 6, 2, 5, 4] if rnd == 0 else [6, 4, 0, 2, 7, 5, 3, 1]
@@ -92,6 +94,7 @@ def test_110m_norms_of_batches_of_eight_against_the_oracle_on_the_full_vectors()
                 v["p"][P - 1] = float("inf")
             base, p = v["base"].cpu().numpy(), v["p"].cpu().numpy()
             want.append(oracle.pg_norm2(base, base, p))
+            plain.alsgd_worker_state_ptrs(w)["p"].copy_(v["p"])
         bases = {ctx.alsgd_worker_state_ptrs(w)["base"].data_ptr() for w in ids}
         assert len(bases) == (8 if rnd == 0 else 1)
         info = ctx.alsgd_arrive(ids, B.ARRIVE_RESEED | B.ARRIVE_NORM | B.ARRIVE_NANCHECK)
@@ -99,5 +102,10 @@ def test_110m_norms_of_batches_of_eight_against_the_oracle_on_the_full_vectors()
             assert got["nonfinite"] == bad == (1 if (rnd == 1 and j == 5) else 0)
             if not bad:
                 assert abs(got["gnorm2"] - norm) <= 1e-6 * norm, (rnd, j, got["gnorm2"], norm)
+        plain.alsgd_arrive(ids, B.ARRIVE_RESEED)
+        for a, b in zip(ctx.alsgd_state_ptrs(), plain.alsgd_state_ptrs()):
+            assert torch.equal(a.view(torch.int32), b.view(torch.int32))
     ctx.alsgd_sync()
+    plain.alsgd_sync()
     ctx.close()
+    plain.close()
